@@ -1,0 +1,193 @@
+/*
+ * ampq.h -- C ABI of the B200 loss-MSE sensitivity pass.
+ *
+ * The library scores every linear layer (operands X, W) and every batched GEMM
+ * (operands X0, X1) of a model over R calibration samples: per-tensor amax and
+ * FP8 scale, round-to-nearest-even FP8 cast, quantisation error, squared error
+ * weighted by the squared loss gradient, per-sample and mean sensitivities; it
+ * then sums the loss-MSE terms per sequential sub-graph and selects the
+ * precision assignment of the paper's integer program under a loss-MSE budget.
+ * Everything up to the per-layer values runs in CUDA kernels on one sm_100a
+ * device; the sub-graph sums and the selection run on the host.
+ *
+ * Conventions
+ *   - Every function returns an int status: AMPQ_OK (0) or a negative
+ *     AMPQ_ERR_* code.  Nothing throws, aborts or prints.  ampq_strerror maps a
+ *     code to text; ampq_last_error(ctx) adds detail for the last failure.
+ *   - "device pointer" = memory of the context's CUDA device; "host pointer" =
+ *     ordinary host memory.  The caller owns every tensor and every output
+ *     array; the library owns only its workspace (tables, per-tile partial
+ *     sums, results), allocated with cudaMalloc when ampq_score first needs it
+ *     and released by ampq_destroy.
+ *   - Kernels are launched on the stream given to ampq_create.  ampq_score is
+ *     asynchronous; the getters synchronise that stream.
+ *   - A context is not thread-safe; use one per thread or lock around it.
+ *   - There is no CPU fallback: without a CUDA device ampq_create fails with
+ *     AMPQ_ERR_CUDA.
+ */
+#ifndef AMPQ_H
+#define AMPQ_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ampq_ctx ampq_ctx;
+
+/* element type of an operand and of its gradient */
+enum { AMPQ_F32 = 0, AMPQ_BF16 = 1 };
+/* numerical formats.  BASE is the high-precision format (BF16 in the paper's
+ * setup, Sec. 3.1); its loss-MSE contribution is 0.  E4M3: 4 exponent, 3
+ * mantissa bits, bias 7, no infinity, largest finite value 448.  E5M2: 5
+ * exponent, 2 mantissa bits, bias 15, largest finite value 57344. */
+enum { AMPQ_FMT_BASE = 0, AMPQ_FMT_E4M3 = 1, AMPQ_FMT_E5M2 = 2 };
+/* layer kinds: Y = X W^T + b (Sec. 2.2, linear layer) and Y = X0 (x) X1 (BGEMM) */
+enum { AMPQ_LINEAR = 0, AMPQ_BGEMM = 1 };
+/* which per-layer loss-MSE feeds the sub-graph sums:
+ * MODEL    d_{l,f} = alpha_f * s_l, alpha_f = 2^(-2 m_f)/12   (Sec. 2.2)
+ * MEASURED d_{l,f} = (1/R) sum_r sum_k (g_k (Q_f(z_k) - z_k))^2, the same
+ *          expectation with the realised FP8 rounding error                */
+enum { AMPQ_D_MODEL = 0, AMPQ_D_MEASURED = 1 };
+/* where a bound tensor lives */
+enum { AMPQ_MEM_DEVICE = 0, AMPQ_MEM_HOST = 1 };
+
+enum {
+    AMPQ_OK = 0,
+    AMPQ_ERR_INVALID = -1,     /* null pointer, bad enum, bad id, bad size          */
+    AMPQ_ERR_ALIGN = -2,       /* a tensor pointer is not aligned to its element    */
+    AMPQ_ERR_STATE = -3,       /* call out of order (e.g. results before a score)   */
+    AMPQ_ERR_CUDA = -4,        /* a CUDA call failed; see ampq_last_error           */
+    AMPQ_ERR_NONFINITE = -5,   /* a scored operand holds Inf or NaN                 */
+    AMPQ_ERR_INFEASIBLE = -6,  /* no assignment meets the budget                    */
+    AMPQ_ERR_TOO_LARGE = -7,   /* selection exceeded its state limit                */
+    AMPQ_ERR_NOMEM = -8
+};
+
+const char *ampq_strerror(int status);
+const char *ampq_last_error(const ampq_ctx *ctx);
+
+/* Creates a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t
+ * (0 = the default stream), borrowed for the life of the context: every kernel
+ * and copy of this context is issued on it. */
+int ampq_create(ampq_ctx **out, int device, void *cuda_stream);
+int ampq_destroy(ampq_ctx *ctx);
+
+/* The F formats of the problem (Sec. 2.1: "F distinct numerical formats").
+ * fmt[0] must be AMPQ_FMT_BASE; fmt[1..F-1] are distinct low-precision formats
+ * (F <= 3).  Default: {BASE, E4M3}.  Must be called before layers are scored;
+ * changing it invalidates earlier results. */
+int ampq_set_formats(ampq_ctx *ctx, const int *fmt, int F);
+
+/* Registers one layer with R calibration samples (Sec. 2.2: layer l, samples
+ * r = 0..R-1).  `name` is copied (may be NULL).  Writes the layer id
+ * (0, 1, 2, ... in registration order). */
+int ampq_register_layer(ampq_ctx *ctx, int kind, const char *name, int R, int *layer_id);
+
+/* Binds operand 0 (X or X0) or 1 (W or X1) of a layer: the two halves of the
+ * layer's extended input z_l (Sec. 2.2).
+ *   values  numel elements of `dtype`, contiguous.
+ *           per_sample_values = 1: laid out [R, numel/R]; sample r owns slice r
+ *           (activations, BGEMM operands; numel must be a multiple of R).
+ *           per_sample_values = 0: one tensor shared by all samples (weights).
+ *   grads   the loss gradient with respect to this operand, same dtype: sample
+ *           r's gradient starts at grads + r*grad_stride elements and has the
+ *           extent of the values it weights (numel/R, or numel when shared).
+ *   mem     AMPQ_MEM_DEVICE: device pointers, read in place.  AMPQ_MEM_HOST:
+ *           host pointers; every ampq_score copies them to library-owned device
+ *           staging on the stream first (pinned memory makes that copy
+ *           asynchronous).
+ * The tensors are borrowed: they must stay valid and unchanged until the work
+ * of the last ampq_score on the stream has finished.  Pointers must be aligned
+ * to the element size (AMPQ_ERR_ALIGN otherwise); 16-byte alignment of every
+ * sample slice enables the vectorised path, anything else is scored
+ * correctly through a slower scalar path.  numel = 0 is allowed (scores 0).
+ * Re-binding replaces the previous binding. */
+int ampq_bind_operand(ampq_ctx *ctx, int layer_id, int operand, int dtype, int mem,
+                      const void *values, long long numel, int per_sample_values,
+                      const void *grads, long long grad_stride);
+
+/* Optional static scale: use `amax` for this operand instead of measuring it
+ * (the amax pass then skips the tensor).  Values above amax saturate.  A
+ * negative amax removes the preset. */
+int ampq_set_amax(ampq_ctx *ctx, int layer_id, int operand, float amax);
+
+/* Scores every layer whose two operands are bound (Algorithm 1 step 2, the
+ * per-element part), asynchronously on the context's stream:
+ *   amax_t = max_k |z_k| per tensor; per format f: scale = fl32(amax/fmax_f),
+ *   inv = fl32(fmax_f/amax) ((1,1) when amax = 0 or inv is not finite);
+ *   q_k = RNE saturating FP8 cast of fl32(z_k * inv); e_k = dec(q_k)*scale - z_k;
+ *   per (tensor, sample): S = sum_k (z_k g_k)^2, D_f = sum_k (g_k e_k)^2;
+ *   per layer: s^r = S(op0,r) + S(op1,r), s = mean_r s^r, d_model_f = alpha_f s,
+ *   d_meas_f = mean_r (D_f(op0,r) + D_f(op1,r)).
+ * Sums are accumulated in fp32 over runs of at most a few hundred terms per
+ * thread and combined in a fixed order in fp64, so results are reproducible
+ * run to run. */
+int ampq_score(ampq_ctx *ctx);
+
+/* Number of kernel launches issued by the last ampq_score (diagnostics). */
+int ampq_last_launch_count(const ampq_ctx *ctx);
+
+/* Results of one layer after ampq_score (synchronises the stream on the first
+ * call after a score).  Any output pointer may be NULL.  Host pointers.
+ *   amax[2]                 per operand
+ *   scale[2*F], inv_scale[2*F]   index operand*F + f; entry f = 0 is 1
+ *   s_per_sample[R]         s_l^r      (Sec. 2.2, per-sample sensitivity)
+ *   s_mean                  s_l        (Sec. 2.2, average sensitivity)
+ *   d_meas_per_sample[R*F]  index r*F + f; column 0 is 0
+ *   d_model[F], d_meas[F]   entry 0 is 0
+ * Returns AMPQ_ERR_NONFINITE if the layer's operands held Inf/NaN. */
+int ampq_get_layer(ampq_ctx *ctx, int layer_id, float *amax, float *scale, float *inv_scale,
+                   double *s_per_sample, double *s_mean, double *d_meas_per_sample,
+                   double *d_model, double *d_meas);
+
+/* Per-operand sums of a layer: out[R*F], index r*F + a, a = 0: S, a = f >= 1:
+ * D_f.  Host pointer. */
+int ampq_get_operand(ampq_ctx *ctx, int layer_id, int operand, double *out);
+
+/* Test hook: writes the FP8 code of every element of a bound DEVICE operand
+ * (numel bytes, device pointer), using the scales of the last ampq_score and
+ * the same cast the scoring kernel applies.  Asynchronous on the stream. */
+int ampq_export_codes(ampq_ctx *ctx, int layer_id, int operand, int fmt, unsigned char *dev_out);
+
+/* Defines sequential sub-graph (group) V_j = {layer_ids[0..Lj-1]} with Pj
+ * configurations (Sec. 2.1): Q[l + Lj*p] in [0,F-1] is the index into the
+ * context's format list that configuration p gives layer l of the group, and
+ * c[p] is its performance metric (time gain, MAC gain or memory gain).  Q and
+ * c are copied.  Writes the group id (0, 1, ... in definition order, which is
+ * also the order j of the selection). */
+int ampq_define_group(ampq_ctx *ctx, const int *layer_ids, int Lj, const unsigned char *Q,
+                      const double *c, int Pj, int *group_id);
+int ampq_clear_groups(ampq_ctx *ctx);
+
+/* d_{j,p} = sum_{l=0}^{Lj-1} d_{l_{j,l}, Q_j[l,p]} (Sec. 2.2, last equation),
+ * left fold in l, from the last score.  d_out[Pj], host pointer. */
+int ampq_group_costs(ampq_ctx *ctx, int group_id, int d_mode, double *d_out);
+
+/* budget = tau^2 * (1/R) sum_r losses[r]^2 (Sec. 2.1; E[g^2] is the
+ * mean-square loss of Algorithm 1 step 2).  Needs no context. */
+int ampq_budget_from_tau(double tau, const double *losses, int R, double *budget);
+
+/* Loss MSE of the configuration that puts every scored layer in format index
+ * f (1..F-1): the left fold over layers of d_{l,f}; used for budgets stated as
+ * a fraction of the all-low-precision loss MSE. */
+int ampq_all_lowp_cost(ampq_ctx *ctx, int d_mode, int f, double *d_all);
+
+/* Solves the integer program of Sec. 2.1 exactly over the defined groups:
+ * maximise sum_j c_{j,p_j} subject to sum_j d_{j,p_j} <= budget, one p_j per
+ * group.  Sums are left folds over j = 0..J-1 in double.  Among optimal
+ * assignments the one with the smaller d wins, then the lexicographically
+ * smaller (p_0..p_{J-1}).  p_out[J] host.  AMPQ_ERR_INFEASIBLE if no
+ * assignment meets the budget. */
+int ampq_select(ampq_ctx *ctx, int d_mode, double budget, int *p_out, double *c_total,
+                double *d_total);
+
+/* The same solver on caller-supplied tables (no context, no GPU): group j owns
+ * entries off[j] .. off[j]+P[j]-1 of c[] and d[]. */
+int ampq_select_tables(int J, const int *P, const long long *off, const double *c,
+                       const double *d, double budget, int *p_out, double *c_total,
+                       double *d_total);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMPQ_H */

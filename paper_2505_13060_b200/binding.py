@@ -1,0 +1,260 @@
+"""Thin ctypes binding of the C-ABI library (``include/ampq.h``).
+
+Argument marshalling only: every step of the scoring path runs in the CUDA
+kernels of ``libampq.so``.  Tensors are passed as raw device (or host)
+pointers; PyTorch is used by callers for device memory and streams.  The
+library must have been built (``python -m paper_2505_13060_b200.build``);
+there is no fallback of any kind, loading fails loudly if it is missing.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libampq.so")
+
+F32, BF16 = 0, 1
+FMT_BASE, FMT_E4M3, FMT_E5M2 = 0, 1, 2
+LINEAR, BGEMM = 0, 1
+D_MODEL, D_MEASURED = 0, 1
+MEM_DEVICE, MEM_HOST = 0, 1
+
+OK = 0
+ERR_INVALID, ERR_ALIGN, ERR_STATE, ERR_CUDA = -1, -2, -3, -4
+ERR_NONFINITE, ERR_INFEASIBLE, ERR_TOO_LARGE, ERR_NOMEM = -5, -6, -7, -8
+
+# every symbol include/ampq.h declares
+EXPORTS = [
+    "ampq_strerror", "ampq_last_error", "ampq_create", "ampq_destroy", "ampq_set_formats",
+    "ampq_register_layer", "ampq_bind_operand", "ampq_set_amax", "ampq_score",
+    "ampq_last_launch_count", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
+    "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
+    "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables",
+]
+
+_lib = None
+
+
+class AmpqError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        msg = lib().ampq_strerror(status).decode()
+        super().__init__("ampq status %d (%s)%s" % (status, msg, (": " + detail) if detail else ""))
+
+
+def lib():
+    """Loads ``libampq.so`` (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "%s is missing: build it with `python -m paper_2505_13060_b200.build` "
+            "(nvcc, sm_100a); there is no fallback path" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i, ll, dp, fp, ip = C.c_void_p, C.c_int, C.c_longlong, C.POINTER(C.c_double), C.POINTER(C.c_float), C.POINTER(C.c_int)
+    L.ampq_strerror.restype = C.c_char_p
+    L.ampq_strerror.argtypes = [i]
+    L.ampq_last_error.restype = C.c_char_p
+    L.ampq_last_error.argtypes = [vp]
+    L.ampq_create.argtypes = [C.POINTER(vp), i, vp]
+    L.ampq_destroy.argtypes = [vp]
+    L.ampq_set_formats.argtypes = [vp, ip, i]
+    L.ampq_register_layer.argtypes = [vp, i, C.c_char_p, i, ip]
+    L.ampq_bind_operand.argtypes = [vp, i, i, i, i, vp, ll, i, vp, ll]
+    L.ampq_set_amax.argtypes = [vp, i, i, C.c_float]
+    L.ampq_score.argtypes = [vp]
+    L.ampq_last_launch_count.argtypes = [vp]
+    L.ampq_get_layer.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.ampq_get_operand.argtypes = [vp, i, i, vp]
+    L.ampq_export_codes.argtypes = [vp, i, i, i, vp]
+    L.ampq_define_group.argtypes = [vp, vp, i, vp, vp, i, ip]
+    L.ampq_clear_groups.argtypes = [vp]
+    L.ampq_group_costs.argtypes = [vp, i, i, vp]
+    L.ampq_budget_from_tau.argtypes = [C.c_double, vp, i, dp]
+    L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
+    L.ampq_select.argtypes = [vp, i, C.c_double, vp, dp, dp]
+    L.ampq_select_tables.argtypes = [i, vp, vp, vp, vp, C.c_double, vp, dp, dp]
+    for name in EXPORTS:
+        if name not in ("ampq_strerror", "ampq_last_error"):
+            getattr(L, name).restype = i
+    _lib = L
+    return L
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def budget_from_tau(tau: float, losses) -> float:
+    g = np.ascontiguousarray(losses, dtype=np.float64)
+    out = C.c_double()
+    rc = lib().ampq_budget_from_tau(tau, _np_ptr(g), g.size, C.byref(out))
+    if rc:
+        raise AmpqError(rc)
+    return out.value
+
+
+def select_tables(c_tables, d_tables, budget: float):
+    """Solves the integer program on explicit tables; returns (p, c, d) or None if infeasible."""
+    P = np.asarray([len(x) for x in c_tables], dtype=np.int32)
+    J = len(P)
+    off = np.zeros(max(J, 1), dtype=np.int64)
+    if J:
+        off[1:J] = np.cumsum(P[:-1])
+    c = np.concatenate([np.asarray(x, np.float64) for x in c_tables]) if J else np.zeros(1)
+    d = np.concatenate([np.asarray(x, np.float64) for x in d_tables]) if J else np.zeros(1)
+    p = np.zeros(max(J, 1), dtype=np.int32)
+    co, do = C.c_double(), C.c_double()
+    rc = lib().ampq_select_tables(J, _np_ptr(P) if J else None, _np_ptr(off), _np_ptr(c), _np_ptr(d),
+                                  budget, _np_ptr(p), C.byref(co), C.byref(do))
+    if rc == ERR_INFEASIBLE:
+        return None
+    if rc:
+        raise AmpqError(rc)
+    return p[:J].copy(), co.value, do.value
+
+
+class Context:
+    """One scoring context on one CUDA device and stream (see ``ampq_create``)."""
+
+    def __init__(self, device: int = 0, stream: int = 0):
+        self._h = C.c_void_p()
+        rc = lib().ampq_create(C.byref(self._h), device, C.c_void_p(stream))
+        if rc:
+            self._h = None
+            raise AmpqError(rc, "ampq_create")
+        self.F = 2
+        self._R = {}
+
+    def _check(self, rc: int):
+        if rc:
+            raise AmpqError(rc, lib().ampq_last_error(self._h).decode())
+
+    def destroy(self):
+        if self._h is not None:
+            lib().ampq_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def set_formats(self, fmts):
+        a = (C.c_int * len(fmts))(*fmts)
+        self._check(lib().ampq_set_formats(self._h, a, len(fmts)))
+        self.F = len(fmts)
+
+    def register_layer(self, kind: int, name: str, R: int) -> int:
+        out = C.c_int()
+        self._check(lib().ampq_register_layer(self._h, kind, name.encode() if name else None, R, C.byref(out)))
+        self._R[out.value] = R
+        return out.value
+
+    def bind_operand(self, layer_id: int, operand: int, dtype: int, values_ptr: int, numel: int,
+                     per_sample_values: bool, grads_ptr: int, grad_stride: int, mem: int = MEM_DEVICE):
+        self._check(lib().ampq_bind_operand(self._h, layer_id, operand, dtype, mem, C.c_void_p(values_ptr),
+                                            numel, 1 if per_sample_values else 0, C.c_void_p(grads_ptr),
+                                            grad_stride))
+
+    def set_amax(self, layer_id: int, operand: int, amax: float):
+        self._check(lib().ampq_set_amax(self._h, layer_id, operand, amax))
+
+    def score(self):
+        self._check(lib().ampq_score(self._h))
+
+    def last_launch_count(self) -> int:
+        return lib().ampq_last_launch_count(self._h)
+
+    def get_layer(self, layer_id: int, allow_nonfinite: bool = False) -> dict:
+        R, F = self._R[layer_id], self.F
+        amax = np.zeros(2, np.float32)
+        scale = np.zeros(2 * F, np.float32)
+        inv = np.zeros(2 * F, np.float32)
+        s_r = np.zeros(R)
+        s_mean = np.zeros(1)
+        d_meas_r = np.zeros(R * F)
+        d_model = np.zeros(F)
+        d_meas = np.zeros(F)
+        rc = lib().ampq_get_layer(self._h, layer_id, _np_ptr(amax), _np_ptr(scale), _np_ptr(inv), _np_ptr(s_r),
+                                  _np_ptr(s_mean), _np_ptr(d_meas_r), _np_ptr(d_model), _np_ptr(d_meas))
+        if rc and not (allow_nonfinite and rc == ERR_NONFINITE):
+            self._check(rc)
+        return dict(amax=amax, scale=scale.reshape(2, F), inv_scale=inv.reshape(2, F), s_per_sample=s_r,
+                    s_mean=float(s_mean[0]), d_meas_per_sample=d_meas_r.reshape(R, F), d_model=d_model,
+                    d_meas=d_meas, status=rc)
+
+    def get_operand(self, layer_id: int, operand: int) -> np.ndarray:
+        out = np.zeros((self._R[layer_id], self.F))
+        self._check(lib().ampq_get_operand(self._h, layer_id, operand, _np_ptr(out)))
+        return out
+
+    def export_codes(self, layer_id: int, operand: int, fmt: int, dev_out_ptr: int):
+        self._check(lib().ampq_export_codes(self._h, layer_id, operand, fmt, C.c_void_p(dev_out_ptr)))
+
+    def define_group(self, layer_ids, Q, c) -> int:
+        """Q: [Lj, Pj] array of format indices (column p = configuration p); c: [Pj]."""
+        ids = np.ascontiguousarray(layer_ids, dtype=np.int32)
+        Q = np.asarray(Q, dtype=np.uint8)
+        Lj, Pj = Q.shape
+        Qf = np.ascontiguousarray(Q.T).reshape(-1)  # Q[l + Lj*p]
+        cc = np.ascontiguousarray(c, dtype=np.float64)
+        assert cc.size == Pj and ids.size == Lj
+        out = C.c_int()
+        self._check(lib().ampq_define_group(self._h, _np_ptr(ids), Lj, _np_ptr(Qf), _np_ptr(cc), Pj, C.byref(out)))
+        if not hasattr(self, "_P"):
+            self._P = {}
+        self._P[out.value] = Pj
+        return out.value
+
+    def clear_groups(self):
+        self._check(lib().ampq_clear_groups(self._h))
+        self._P = {}
+
+    def group_costs(self, group_id: int, d_mode: int = D_MODEL) -> np.ndarray:
+        out = np.zeros(self._P[group_id])
+        self._check(lib().ampq_group_costs(self._h, group_id, d_mode, _np_ptr(out)))
+        return out
+
+    def all_lowp_cost(self, d_mode: int, f: int) -> float:
+        out = C.c_double()
+        self._check(lib().ampq_all_lowp_cost(self._h, d_mode, f, C.byref(out)))
+        return out.value
+
+    def select(self, d_mode: int, budget: float):
+        """Returns (p[J], c_total, d_total), or None when no assignment meets the budget."""
+        J = len(getattr(self, "_P", {}))
+        p = np.zeros(max(J, 1), dtype=np.int32)
+        co, do = C.c_double(), C.c_double()
+        rc = lib().ampq_select(self._h, d_mode, budget, _np_ptr(p), C.byref(co), C.byref(do))
+        if rc == ERR_INFEASIBLE:
+            return None
+        self._check(rc)
+        return p[:J].copy(), co.value, do.value
+
+
+def torch_dtype_code(t) -> int:
+    import torch
+
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("operands are float32 or bfloat16, got %s" % t.dtype)
+
+
+def bind_layer_tensors(ctx: Context, layer_id: int, lt, mem: int = MEM_DEVICE):
+    """Binds both operands of a ``synth.LayerTensors`` (or anything with
+    ``spec``, ``values`` and ``grads`` laid out the same way)."""
+    R = lt.spec.R
+    for k, op in enumerate((lt.spec.op0, lt.spec.op1)):
+        v, g = lt.values[k], lt.grads[k]
+        assert v.is_contiguous() and g.is_contiguous()
+        ext = v.numel() // R if op.per_sample else v.numel()
+        ctx.bind_operand(layer_id, k, torch_dtype_code(v), v.data_ptr(), v.numel(), op.per_sample,
+                         g.data_ptr(), ext, mem)

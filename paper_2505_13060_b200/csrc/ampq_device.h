@@ -1,0 +1,59 @@
+// Device-side tables shared by the kernels (ampq_kernels.cu) and the host
+// library (ampq_lib.cu).  Plain structs, no torch types.
+#pragma once
+#include <cstdint>
+
+namespace ampq {
+
+constexpr int kThreads = 256;          // threads per CTA in every streaming kernel
+constexpr int kTileElems = 32768;      // elements of one tile (one CTA's unit of work)
+constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
+constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
+constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
+
+// internal low-precision slots: bit 0 = E4M3, bit 1 = E5M2.  With both present
+// slot 0 is E4M3 and slot 1 is E5M2; with one present it is slot 0.
+constexpr int kMaskE4M3 = 1;
+constexpr int kMaskE5M2 = 2;
+
+// One bound operand of a scored layer.
+struct Tensor {
+    const void* values;      // device pointer, numel elements
+    const void* grads;       // device pointer; sample r at grads + r*grad_stride
+    long long numel;         // value elements in total
+    long long seg_len;       // elements of one segment: numel/R (per-sample) or numel (shared)
+    long long grad_stride;   // elements between consecutive samples' gradients
+    long long partial_base;  // partial slot of (r, i) = partial_base + r*tiles_per_seg + i
+    int tiles_per_seg;       // ceil(seg_len / kTileElems)
+    int R;                   // calibration samples
+    int per_sample;          // 1: values are [R, seg_len]; 0: shared by all samples
+    int dtype;               // AMPQ_F32 / AMPQ_BF16
+    int rgroups;             // shared values: ceil(R / kMaxRB) tiles per value tile; else 1
+    int seg_base;            // index of segment (this tensor, r = 0) in the segment outputs
+    float amax_preset;       // >= 0: use instead of measuring
+    int pad;
+};
+
+// One segment = (tensor, sample): its partial slots are contiguous.
+struct Segment {
+    long long first_slot;
+    int count;
+    int pad;
+};
+
+// One scored layer for the combine step.
+struct Layer {
+    int seg_base0, seg_base1;  // segment index of (operand, r = 0)
+    int tensor0, tensor1;
+    int R;
+    int out_off;               // offset (doubles) of this layer's block in the layer outputs
+};
+
+// Layer output block layout (doubles): s_r[R], s_mean, d_meas_r[R*F], d_model[F], d_meas[F]
+inline int layer_block_doubles(int R, int F) { return R + 1 + R * F + 2 * F; }
+
+struct LaunchStatus {
+    int nonfinite;  // set when some tensor's amax is Inf/NaN
+};
+
+}  // namespace ampq

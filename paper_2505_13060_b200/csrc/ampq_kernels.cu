@@ -1,0 +1,567 @@
+// CUDA kernels of the loss-MSE sensitivity pass for sm_100a.
+//
+// The pass is a stream-reduce: every operand element and its gradient are read
+// once from HBM, all arithmetic happens in registers, and a few floats per
+// 32768-element tile are written back.  The kernels are therefore shaped for
+// HBM bandwidth: 128-bit coalesced non-allocating loads, several independent
+// loads in flight per thread, packed two-wide fp32 arithmetic (fma.rn.f32x2)
+// and the hardware FP8 converts so that the instruction count per element stays
+// below what 148 SMs can issue at full memory speed.  No tensor cores: there is
+// no contraction anywhere on this path.
+//
+//   amax_kernel     max_k |z_k| per tensor (integer max of the bit patterns,
+//                   warp redux + one atomicMax per CTA)
+//   scales_kernel   scale = amax/fmax, inv = fmax/amax per tensor and format
+//   score_kernel    fused cast / error / weighting / per-tile reduction
+//   finalize_kernel ordered fp64 sum of the per-tile partials per segment
+//   combine_kernel  per-layer sensitivities and loss-MSE terms (Sec. 2.2)
+//   codes_kernel    test hook: the FP8 codes the scoring kernel sees
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cstdint>
+
+#include "ampq_device.h"
+#include "ampq_kernels.h"
+
+namespace ampq {
+
+// ---------------------------------------------------------------------------
+// small device helpers
+
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// Two fp32 values -> two FP8 codes (round to nearest even, saturate to the
+// largest finite value), first argument in the low byte.
+template <int FMT>
+__device__ __forceinline__ unsigned short cast_pair(float lo, float hi) {
+    unsigned short r;
+    if (FMT == kMaskE4M3)
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    else
+        asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Two FP8 codes -> their exact values as fp32 (every FP8 value is an fp16 value).
+template <int FMT>
+__device__ __forceinline__ float2 decode_pair(unsigned short c) {
+    unsigned h;
+    if (FMT == kMaskE4M3)
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h) : "h"(c));
+    else
+        asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h) : "h"(c));
+    __half2 hh = *reinterpret_cast<__half2*>(&h);
+    return __half22float2(hh);
+}
+
+// -(dec(Q(z*inv))*scale - z) for a pair: the negated quantisation error; only
+// its square is used.  One fp32 rounding in y = z*inv, one in the fma.
+template <int FMT>
+__device__ __forceinline__ float2 neg_err_pair(float2 z, float2 inv2, float2 nscale2) {
+    float2 y = __fmul2_rn(z, inv2);
+    float2 dq = decode_pair<FMT>(cast_pair<FMT>(y.x, y.y));
+    return __ffma2_rn(dq, nscale2, z);
+}
+
+template <int DT>
+struct Elem;
+template <>
+struct Elem<0> {  // fp32
+    static constexpr int kPerVec = 4;
+    static constexpr int kBytes = 4;
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&out)[2]) {
+        out[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        out[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+    }
+    __device__ static __forceinline__ float load(const void* p, long long i) {
+        return __ldg(reinterpret_cast<const float*>(p) + i);
+    }
+};
+template <>
+struct Elem<1> {  // bf16: the upper half of an fp32
+    static constexpr int kPerVec = 8;
+    static constexpr int kBytes = 2;
+    __device__ static __forceinline__ float2 two(unsigned w) {
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    }
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&out)[4]) {
+        out[0] = two(v.x); out[1] = two(v.y); out[2] = two(v.z); out[3] = two(v.w);
+    }
+    __device__ static __forceinline__ float load(const void* p, long long i) {
+        unsigned short b = __ldg(reinterpret_cast<const unsigned short*>(p) + i);
+        return __uint_as_float(static_cast<unsigned>(b) << 16);
+    }
+};
+
+// Which tensor owns global tile `tile`: begin[j] <= tile < begin[j+1].  All
+// threads of the CTA take part; the answer is broadcast through shared memory.
+__device__ __forceinline__ int find_tensor(const long long* __restrict__ begin, int T,
+                                           long long tile, int* s_slot) {
+    for (int j = threadIdx.x; j < T; j += blockDim.x) {
+        if (tile >= __ldg(begin + j) && tile < __ldg(begin + j + 1)) *s_slot = j;
+    }
+    __syncthreads();
+    return *s_slot;
+}
+
+// ---------------------------------------------------------------------------
+// amax
+
+__global__ void init_amax_kernel(const Tensor* __restrict__ tens, int T,
+                                 unsigned* __restrict__ amax_bits, LaunchStatus* status) {
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t == 0) status->nonfinite = 0;
+    if (t < T) {
+        float p = tens[t].amax_preset;
+        amax_bits[t] = (p >= 0.0f) ? __float_as_uint(p) : 0u;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
+            unsigned* __restrict__ amax_bits) {
+    __shared__ int s_slot;
+    __shared__ unsigned s_warp[kThreads / 32];
+    const long long tile = blockIdx.x;
+    const int t = find_tensor(tile_begin, T, tile, &s_slot);
+    const Tensor& tn = tens[t];
+    const long long first = (tile - __ldg(tile_begin + t)) * (long long)kTileElems;
+    const long long left = tn.numel - first;
+    const int n = left < kTileElems ? (int)left : kTileElems;
+    const int es = tn.dtype == 0 ? 4 : 2;
+    const char* base = reinterpret_cast<const char*>(tn.values) + first * es;
+    unsigned m = 0;  // fp32 bit pattern of the running max |x|
+    if ((reinterpret_cast<uintptr_t>(base) & 15) == 0) {
+        const int per = 16 / es;
+        const int nvec = n / per;
+        const uint4* vp = reinterpret_cast<const uint4*>(base);
+        if (tn.dtype == 0) {
+            for (int i = threadIdx.x; i < nvec; i += kThreads * 4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    int idx = i + u * kThreads;
+                    v[u] = idx < nvec ? ld_stream_v4(vp + idx) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    m = max(m, v[u].x & 0x7FFFFFFFu); m = max(m, v[u].y & 0x7FFFFFFFu);
+                    m = max(m, v[u].z & 0x7FFFFFFFu); m = max(m, v[u].w & 0x7FFFFFFFu);
+                }
+            }
+        } else {
+            unsigned lo = 0, hi = 0;  // 16-bit patterns of |x|
+            for (int i = threadIdx.x; i < nvec; i += kThreads * 4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    int idx = i + u * kThreads;
+                    v[u] = idx < nvec ? ld_stream_v4(vp + idx) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        lo = max(lo, w[k] & 0x7FFFu);
+                        hi = max(hi, w[k] & 0x7FFF0000u);
+                    }
+                }
+            }
+            m = max(lo << 16, hi);
+        }
+        for (int i = nvec * per + threadIdx.x; i < n; i += kThreads) {
+            float x = tn.dtype == 0 ? Elem<0>::load(base, i) : Elem<1>::load(base, i);
+            m = max(m, __float_as_uint(x) & 0x7FFFFFFFu);
+        }
+    } else {
+        for (int i = threadIdx.x; i < n; i += kThreads) {
+            float x = tn.dtype == 0 ? Elem<0>::load(base, i) : Elem<1>::load(base, i);
+            m = max(m, __float_as_uint(x) & 0x7FFFFFFFu);
+        }
+    }
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned r = s_warp[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) r = max(r, s_warp[w]);
+        atomicMax(amax_bits + t, r);
+    }
+}
+
+// scale = fl32(amax / fmax), inv = fl32(fmax / amax), IEEE divisions; the
+// neutral pair (1, 1) when amax is 0 or fmax/amax is not a finite fp32.
+__global__ void scales_kernel(int T, int fmask, const unsigned* __restrict__ amax_bits,
+                              float* __restrict__ scales, int* __restrict__ tensor_flags,
+                              LaunchStatus* status) {
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    unsigned bits = amax_bits[t];
+    int bad = bits >= 0x7F800000u;
+    tensor_flags[t] = bad;
+    if (bad) atomicExch(&status->nonfinite, 1);
+    float amax = __uint_as_float(bits);
+    int slot = 0;
+#pragma unroll
+    for (int f = 1; f <= 2; ++f) {
+        if (!(fmask & f)) continue;
+        float fmax = (f == kMaskE4M3) ? 448.0f : 57344.0f;
+        float scale = 1.0f, inv = 1.0f;
+        if (!bad && amax > 0.0f) {
+            float i = __fdiv_rn(fmax, amax);
+            if (i <= 3.402823466e+38f) {
+                inv = i;
+                scale = __fdiv_rn(amax, fmax);
+            }
+        }
+        scales[t * 2 * kMaxLow + slot * 2 + 0] = scale;
+        scales[t * 2 * kMaxLow + slot * 2 + 1] = inv;
+        ++slot;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// fused scoring
+
+template <int FMASK>
+struct Fm {
+    static constexpr int kLow = (FMASK & 1) + ((FMASK >> 1) & 1);
+    static constexpr int kAcc = 1 + kLow;
+    static constexpr int kFmt0 = (FMASK & 1) ? kMaskE4M3 : kMaskE5M2;
+    static constexpr int kFmt1 = kMaskE5M2;
+};
+
+// Accumulators of one sample: S and D per low format, two fp32 lanes each.
+template <int NACC>
+struct Acc {
+    float2 v[NACC];
+};
+
+template <int FMASK, int RB, int NP>
+__device__ __forceinline__ void accumulate_pairs(const float2 (&z)[NP], const float2 (&g)[RB][NP],
+                                                 const float2 (&inv2)[2], const float2 (&nsc2)[2],
+                                                 Acc<Fm<FMASK>::kAcc> (&acc)[RB]) {
+#pragma unroll
+    for (int k = 0; k < NP; ++k) {
+        float2 ne0 = neg_err_pair<Fm<FMASK>::kFmt0>(z[k], inv2[0], nsc2[0]);
+        float2 ne1;
+        if constexpr (Fm<FMASK>::kLow == 2) ne1 = neg_err_pair<Fm<FMASK>::kFmt1>(z[k], inv2[1], nsc2[1]);
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            float2 p = __fmul2_rn(z[k], g[r][k]);
+            acc[r].v[0] = __ffma2_rn(p, p, acc[r].v[0]);
+            float2 t0 = __fmul2_rn(ne0, g[r][k]);
+            acc[r].v[1] = __ffma2_rn(t0, t0, acc[r].v[1]);
+            if constexpr (Fm<FMASK>::kLow == 2) {
+                float2 t1 = __fmul2_rn(ne1, g[r][k]);
+                acc[r].v[Fm<FMASK>::kAcc - 1] = __ffma2_rn(t1, t1, acc[r].v[Fm<FMASK>::kAcc - 1]);
+            }
+        }
+    }
+}
+
+// One tile: n elements of values at vbase weighted by RB gradient streams.
+template <int DT, int FMASK, int RB>
+__device__ __forceinline__ void score_tile(const char* vbase, const char* const (&gbase)[RB], int n,
+                                           const float2 (&inv2)[2], const float2 (&nsc2)[2],
+                                           Acc<Fm<FMASK>::kAcc> (&acc)[RB]) {
+    using E = Elem<DT>;
+    constexpr int NP = E::kPerVec / 2;
+    constexpr int U = RB == 1 ? 4 : (RB == 2 ? 2 : 1);
+    bool aligned = (reinterpret_cast<uintptr_t>(vbase) & 15) == 0;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) aligned = aligned && (reinterpret_cast<uintptr_t>(gbase[r]) & 15) == 0;
+    int done = 0;
+    if (aligned) {
+        const int nvec = n / E::kPerVec;
+        const uint4* vp = reinterpret_cast<const uint4*>(vbase);
+        for (int i = threadIdx.x; i < nvec; i += kThreads * U) {
+            uint4 v[U], g[RB][U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int idx = i + u * kThreads;
+                if (idx < nvec) {
+                    v[u] = ld_stream_v4(vp + idx);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+                        g[r][u] = ld_stream_v4(reinterpret_cast<const uint4*>(gbase[r]) + idx);
+                } else {  // zeros add nothing to any sum
+                    v[u] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r) g[r][u] = make_uint4(0, 0, 0, 0);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float2 z[NP], gg[RB][NP];
+                E::unpack(v[u], z);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) E::unpack(g[r][u], gg[r]);
+                accumulate_pairs<FMASK, RB, NP>(z, gg, inv2, nsc2, acc);
+            }
+        }
+        done = nvec * E::kPerVec;
+    }
+    // ragged tail of an aligned tile, or the whole of a misaligned one
+    for (int i = done + threadIdx.x; i < n; i += kThreads) {
+        float2 z[1], gg[RB][1];
+        z[0] = make_float2(E::load(vbase, i), 0.0f);
+#pragma unroll
+        for (int r = 0; r < RB; ++r) gg[r][0] = make_float2(E::load(gbase[r], i), 0.0f);
+        accumulate_pairs<FMASK, RB, 1>(z, gg, inv2, nsc2, acc);
+    }
+}
+
+// CTA-wide sum of RB*NACC values in a fixed order; thread a < RB*NACC writes
+// partial (r, a) of the tile.
+template <int NACC, int RB>
+__device__ __forceinline__ void reduce_and_store(Acc<NACC> (&acc)[RB], float* s_red,
+                                                 float* __restrict__ partials, long long slot0,
+                                                 long long slot_stride) {
+    constexpr int NV = RB * NACC;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+#pragma unroll
+        for (int a = 0; a < NACC; ++a) {
+            float x = acc[r].v[a].x + acc[r].v[a].y;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+            if (lane == 0) s_red[warp * NV + r * NACC + a] = x;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < NV) {
+        float x = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) x += s_red[w * NV + threadIdx.x];
+        const int r = threadIdx.x / NACC, a = threadIdx.x % NACC;
+        partials[(slot0 + r * slot_stride) * NACC + a] = x;
+    }
+}
+
+template <int DT, int FMASK, int RB>
+__device__ __forceinline__ void score_tile_and_store(const Tensor& tn, long long voff, long long goff,
+                                                     int r0, int n, const float2 (&inv2)[2],
+                                                     const float2 (&nsc2)[2], float* s_red,
+                                                     float* __restrict__ partials, long long slot0) {
+    constexpr int NACC = Fm<FMASK>::kAcc;
+    Acc<NACC> acc[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
+#pragma unroll
+        for (int a = 0; a < NACC; ++a) acc[r].v[a] = make_float2(0.0f, 0.0f);
+    const int es = Elem<DT>::kBytes;
+    const char* vbase = reinterpret_cast<const char*>(tn.values) + voff * es;
+    const char* gbase[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
+        gbase[r] = reinterpret_cast<const char*>(tn.grads) + (goff + (long long)(r0 + r) * tn.grad_stride) * es;
+    score_tile<DT, FMASK, RB>(vbase, gbase, n, inv2, nsc2, acc);
+    reduce_and_store<NACC, RB>(acc, s_red, partials, slot0, tn.tiles_per_seg);
+}
+
+template <int FMASK>
+__global__ void __launch_bounds__(kThreads)
+score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
+             const float* __restrict__ scales, float* __restrict__ partials) {
+    __shared__ int s_slot;
+    __shared__ float s_red[(kThreads / 32) * kMaxRB * kMaxAcc];
+    const long long tile = blockIdx.x;
+    const int t = find_tensor(tile_begin, T, tile, &s_slot);
+    const Tensor& tn = tens[t];
+    const int local = (int)(tile - __ldg(tile_begin + t));
+    float2 inv2[2], nsc2[2];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+        float sc = __ldg(scales + t * 2 * kMaxLow + s * 2 + 0);
+        float iv = __ldg(scales + t * 2 * kMaxLow + s * 2 + 1);
+        inv2[s] = make_float2(iv, iv);
+        nsc2[s] = make_float2(-sc, -sc);
+    }
+    int i, r0, rb;  // value tile within the segment, first sample, samples in this tile
+    long long voff;
+    if (tn.per_sample) {
+        r0 = local / tn.tiles_per_seg;
+        i = local - r0 * tn.tiles_per_seg;
+        rb = 1;
+        voff = (long long)r0 * tn.seg_len + (long long)i * kTileElems;
+    } else {
+        i = local / tn.rgroups;
+        r0 = (local - i * tn.rgroups) * kMaxRB;
+        rb = min(kMaxRB, tn.R - r0);
+        voff = (long long)i * kTileElems;
+    }
+    const long long goff = (long long)i * kTileElems;  // offset inside a sample's gradient
+    const long long left = tn.seg_len - (long long)i * kTileElems;
+    const int n = left < kTileElems ? (int)left : kTileElems;
+    const long long slot0 = tn.partial_base + (long long)r0 * tn.tiles_per_seg + i;
+#define AMPQ_TILE(DT, RB) \
+    score_tile_and_store<DT, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0)
+    if (tn.dtype == 0) {
+        switch (rb) {
+            case 1: AMPQ_TILE(0, 1); break;
+            case 2: AMPQ_TILE(0, 2); break;
+            case 3: AMPQ_TILE(0, 3); break;
+            default: AMPQ_TILE(0, 4); break;
+        }
+    } else {
+        switch (rb) {
+            case 1: AMPQ_TILE(1, 1); break;
+            case 2: AMPQ_TILE(1, 2); break;
+            case 3: AMPQ_TILE(1, 3); break;
+            default: AMPQ_TILE(1, 4); break;
+        }
+    }
+#undef AMPQ_TILE
+}
+
+// ---------------------------------------------------------------------------
+// ordered fp64 combine of the per-tile partials: one warp per segment, lane j
+// sums slots j, j+32, ... in order, then a fixed shuffle tree.
+__global__ void finalize_kernel(const Segment* __restrict__ segs, int nseg, int nacc,
+                                const float* __restrict__ partials, double* __restrict__ seg_out) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= nseg) return;
+    const Segment sg = segs[warp];
+    for (int a = 0; a < nacc; ++a) {
+        double x = 0.0;
+        for (int j = lane; j < sg.count; j += 32) x += (double)partials[(sg.first_slot + j) * nacc + a];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+        if (lane == 0) seg_out[(long long)warp * nacc + a] = x;
+    }
+}
+
+// Per layer (Sec. 2.2): s^r = S(op0,r) + S(op1,r); s = (1/R) sum_r s^r;
+// d_model_f = alpha_f s; d_meas^r_f = D_f(op0,r) + D_f(op1,r); d_meas_f = mean_r.
+// Format index f = 0 is the high-precision baseline and costs 0.
+__global__ void combine_kernel(const Layer* __restrict__ layers, int L, int F, CombineParams prm,
+                               const double* __restrict__ seg_out, double* __restrict__ layer_out) {
+    int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= L) return;
+    const Layer ly = layers[l];
+    const int nacc = prm.nacc, R = ly.R;
+    double* o = layer_out + ly.out_off;
+    double* s_r = o;
+    double* s_mean = o + R;
+    double* d_meas_r = o + R + 1;
+    double* d_model = d_meas_r + (long long)R * F;
+    double* d_meas = d_model + F;
+    double acc = 0.0;
+    for (int r = 0; r < R; ++r) {
+        double v = seg_out[(long long)(ly.seg_base0 + r) * nacc] + seg_out[(long long)(ly.seg_base1 + r) * nacc];
+        s_r[r] = v;
+        acc += v;
+    }
+    const double sm = acc / (double)R;
+    *s_mean = sm;
+    d_model[0] = 0.0;
+    d_meas[0] = 0.0;
+    for (int r = 0; r < R; ++r) d_meas_r[(long long)r * F] = 0.0;
+    for (int f = 1; f < F; ++f) {
+        const int a = prm.acc_of_fmt[f];
+        d_model[f] = prm.alpha[f] * sm;
+        double s = 0.0;
+        for (int r = 0; r < R; ++r) {
+            double v = seg_out[(long long)(ly.seg_base0 + r) * nacc + a] +
+                       seg_out[(long long)(ly.seg_base1 + r) * nacc + a];
+            d_meas_r[(long long)r * F + f] = v;
+            s += v;
+        }
+        d_meas[f] = s / (double)R;
+    }
+}
+
+// Test hook: codes of n elements with the scoring kernel's own cast.
+template <int DT, int FMT>
+__global__ void codes_kernel(const void* __restrict__ values, long long n, const float* __restrict__ scale_pair,
+                             unsigned char* __restrict__ out) {
+    const float inv = scale_pair[1];
+    const long long npairs = (n + 1) / 2;
+    for (long long p = blockIdx.x * (long long)blockDim.x + threadIdx.x; p < npairs;
+         p += (long long)gridDim.x * blockDim.x) {
+        const long long i = 2 * p;
+        float2 z = make_float2(Elem<DT>::load(values, i), i + 1 < n ? Elem<DT>::load(values, i + 1) : 0.0f);
+        float2 y = __fmul2_rn(z, make_float2(inv, inv));
+        unsigned short c = cast_pair<FMT>(y.x, y.y);
+        out[i] = (unsigned char)(c & 0xFF);
+        if (i + 1 < n) out[i + 1] = (unsigned char)(c >> 8);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host launchers
+
+cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, LaunchStatus* status,
+                             cudaStream_t st) {
+    init_amax_kernel<<<(T + 255) / 256 > 0 ? (T + 255) / 256 : 1, 256, 0, st>>>(tens, T, amax_bits, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                        unsigned* amax_bits, cudaStream_t st) {
+    if (ntiles <= 0) return cudaSuccess;
+    amax_kernel<<<(unsigned)ntiles, kThreads, 0, st>>>(tens, tile_begin, T, amax_bits);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
+                          LaunchStatus* status, cudaStream_t st) {
+    if (T <= 0) return cudaSuccess;
+    scales_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, fmask, amax_bits, scales, tensor_flags, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_score(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int fmask,
+                         const float* scales, float* partials, cudaStream_t st) {
+    if (ntiles <= 0) return cudaSuccess;
+    const unsigned grid = (unsigned)ntiles;
+    switch (fmask) {
+        case 1: score_kernel<1><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        case 2: score_kernel<2><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        case 3: score_kernel<3><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const float* partials, double* seg_out,
+                            cudaStream_t st) {
+    if (nseg <= 0) return cudaSuccess;
+    const int warps_per_block = 8;
+    finalize_kernel<<<(nseg + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+        segs, nseg, nacc, partials, seg_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParams& prm, const double* seg_out,
+                           double* layer_out, cudaStream_t st) {
+    if (L <= 0) return cudaSuccess;
+    combine_kernel<<<(L + 127) / 128, 128, 0, st>>>(layers, L, F, prm, seg_out, layer_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_codes(int dtype, int fmt_mask, const void* values, long long n, const float* scale_pair,
+                         unsigned char* out, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    long long blocks = ((n + 1) / 2 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    const unsigned grid = (unsigned)blocks;
+    if (dtype == 0 && fmt_mask == kMaskE4M3) codes_kernel<0, kMaskE4M3><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else if (dtype == 0) codes_kernel<0, kMaskE5M2><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else if (fmt_mask == kMaskE4M3) codes_kernel<1, kMaskE4M3><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else codes_kernel<1, kMaskE5M2><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    return cudaGetLastError();
+}
+
+}  // namespace ampq

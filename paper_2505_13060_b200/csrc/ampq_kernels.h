@@ -1,0 +1,32 @@
+// Host-callable launchers of the kernels in ampq_kernels.cu.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "ampq_device.h"
+
+namespace ampq {
+
+// alpha[f] = 2^(-2 m_f)/12 of user format index f (entry 0 unused: the baseline
+// costs 0); acc_of_fmt[f] = accumulator column (1 or 2) holding D of format f.
+struct CombineParams {
+    double alpha[1 + kMaxLow];
+    int acc_of_fmt[1 + kMaxLow];
+    int nacc;
+};
+
+cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, LaunchStatus* status,
+                             cudaStream_t st);
+cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                        unsigned* amax_bits, cudaStream_t st);
+cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
+                          LaunchStatus* status, cudaStream_t st);
+cudaError_t launch_score(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int fmask,
+                         const float* scales, float* partials, cudaStream_t st);
+cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const float* partials, double* seg_out,
+                            cudaStream_t st);
+cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParams& prm, const double* seg_out,
+                           double* layer_out, cudaStream_t st);
+cudaError_t launch_codes(int dtype, int fmt_mask, const void* values, long long n, const float* scale_pair,
+                         unsigned char* out, cudaStream_t st);
+
+}  // namespace ampq

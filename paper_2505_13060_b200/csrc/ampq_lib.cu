@@ -1,0 +1,714 @@
+// C ABI of the sensitivity pass (include/ampq.h): registry of layers, operands
+// and groups, the device work tables, the launch sequence, result read-back,
+// sub-graph sums and the selection call.  Host code; the arithmetic of the hot
+// path is in ampq_kernels.cu.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/ampq.h"
+#include "ampq_device.h"
+#include "ampq_kernels.h"
+#include "ampq_select.h"
+
+using namespace ampq;
+
+namespace {
+
+struct Operand {
+    bool bound = false;
+    int dtype = 0, mem = 0, per_sample = 0;
+    const void* values = nullptr;
+    const void* grads = nullptr;
+    long long numel = 0, grad_stride = 0;
+    float amax_preset = -1.0f;
+    void* stage = nullptr;  // device staging for host-bound operands
+    size_t stage_bytes = 0;
+    int tensor = -1;        // index in the tables of the last score, or -1
+};
+
+struct LayerRec {
+    int kind = 0, R = 1;
+    std::string name;
+    Operand op[2];
+    int scored = -1;  // index among the layers of the last score, or -1
+};
+
+struct Group {
+    std::vector<int> layers;
+    std::vector<unsigned char> Q;
+    std::vector<double> c;
+    int P = 0;
+};
+
+template <typename T>
+struct DevBuf {
+    T* p = nullptr;
+    size_t cap = 0;
+    cudaError_t ensure(size_t n) {
+        if (n <= cap) return cudaSuccess;
+        if (p) cudaFree(p);
+        p = nullptr;
+        cap = 0;
+        size_t want = n + n / 4 + 16;
+        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&p), want * sizeof(T));
+        if (e == cudaSuccess) cap = want;
+        return e;
+    }
+    void release() {
+        if (p) cudaFree(p);
+        p = nullptr;
+        cap = 0;
+    }
+};
+
+template <typename T>
+struct PinBuf {
+    T* p = nullptr;
+    size_t cap = 0;
+    cudaError_t ensure(size_t n) {
+        if (n <= cap) return cudaSuccess;
+        if (p) cudaFreeHost(p);
+        p = nullptr;
+        cap = 0;
+        size_t want = n + n / 4 + 16;
+        cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&p), want * sizeof(T));
+        if (e == cudaSuccess) cap = want;
+        return e;
+    }
+    void release() {
+        if (p) cudaFreeHost(p);
+        p = nullptr;
+        cap = 0;
+    }
+};
+
+int mantissa_bits_of(int fmt) { return fmt == AMPQ_FMT_E4M3 ? 3 : (fmt == AMPQ_FMT_E5M2 ? 2 : 7); }
+
+}  // namespace
+
+struct ampq_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int F = 2;
+    int fmt[1 + kMaxLow] = {AMPQ_FMT_BASE, AMPQ_FMT_E4M3, 0};
+    int fmask = kMaskE4M3;
+    int slot_of_fmt[1 + kMaxLow] = {-1, 0, -1};  // user format index -> internal low slot
+    std::vector<LayerRec> layers;
+    std::vector<Group> groups;
+    bool dirty = true;     // bindings changed since the tables were built
+    bool scored = false;   // a score has been issued
+    bool pending = false;  // its results have not been synchronised yet
+    int launches = 0;
+    std::string err;
+
+    // tables of the last score (host copies)
+    std::vector<Tensor> tens;
+    std::vector<long long> tile_begin, amax_tile_begin;
+    std::vector<Segment> segs;
+    std::vector<Layer> lay;
+    std::vector<int> scored_layer_ids;
+    long long ntiles = 0, namax_tiles = 0, nslots = 0;
+    int layer_out_doubles = 0;
+
+    DevBuf<Tensor> d_tens;
+    DevBuf<long long> d_tile_begin, d_amax_tile_begin;
+    DevBuf<Segment> d_segs;
+    DevBuf<Layer> d_lay;
+    DevBuf<unsigned> d_amax_bits;
+    DevBuf<float> d_scales, d_partials;
+    DevBuf<int> d_flags;
+    DevBuf<double> d_seg_out, d_layer_out;
+    DevBuf<LaunchStatus> d_status;
+    PinBuf<unsigned> h_amax_bits;
+    PinBuf<float> h_scales;
+    PinBuf<int> h_flags;
+    PinBuf<double> h_seg_out, h_layer_out;
+    PinBuf<LaunchStatus> h_status;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+int fail(ampq_ctx* ctx, int code, const std::string& msg) {
+    if (ctx) ctx->err = msg;
+    return code;
+}
+
+int cuda_fail(ampq_ctx* ctx, cudaError_t e, const char* where) {
+    if (ctx) ctx->err = std::string(where) + ": " + cudaGetErrorString(e);
+    return AMPQ_ERR_CUDA;
+}
+
+#define AMPQ_CUDA(call, where)                         \
+    do {                                               \
+        cudaError_t e__ = (call);                      \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, where); \
+    } while (0)
+
+bool layer_ready(const LayerRec& l) { return l.op[0].bound && l.op[1].bound; }
+
+long long extent_of(const LayerRec& l, const Operand& o) { return o.per_sample ? o.numel / l.R : o.numel; }
+
+// Builds the host tables for every layer whose two operands are bound.
+int build_tables(ampq_ctx* ctx) {
+    ctx->tens.clear(); ctx->tile_begin.clear(); ctx->amax_tile_begin.clear();
+    ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
+    for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
+    long long tiles = 0, atiles = 0, slots = 0;
+    int out_off = 0;
+    for (size_t li = 0; li < ctx->layers.size(); ++li) {
+        LayerRec& l = ctx->layers[li];
+        if (!layer_ready(l)) continue;
+        Layer ly{};
+        ly.R = l.R;
+        ly.out_off = out_off;
+        out_off += layer_block_doubles(l.R, ctx->F);
+        for (int k = 0; k < 2; ++k) {
+            Operand& o = l.op[k];
+            Tensor t{};
+            const long long ext = extent_of(l, o);
+            const int es = o.dtype == AMPQ_F32 ? 4 : 2;
+            if (o.mem == AMPQ_MEM_HOST) {
+                // staging: values, then R gradient slices back to back
+                const size_t vbytes = (((size_t)o.numel * es) + 255) / 256 * 256;  // keeps the gradients 256-byte aligned
+                const size_t need = vbytes + (size_t)l.R * ext * es;
+                if (need > o.stage_bytes) {
+                    if (o.stage) cudaFree(o.stage);
+                    o.stage = nullptr; o.stage_bytes = 0;
+                    if (need) {
+                        AMPQ_CUDA(cudaMalloc(&o.stage, need), "cudaMalloc(staging)");
+                        o.stage_bytes = need;
+                    }
+                }
+                t.values = o.stage;
+                t.grads = reinterpret_cast<const char*>(o.stage) + vbytes;
+                t.grad_stride = ext;
+            } else {
+                t.values = o.values;
+                t.grads = o.grads;
+                t.grad_stride = o.grad_stride;
+            }
+            t.numel = o.numel;
+            t.seg_len = ext;
+            t.R = l.R;
+            t.per_sample = o.per_sample;
+            t.dtype = o.dtype;
+            t.tiles_per_seg = (int)((ext + kTileElems - 1) / kTileElems);
+            t.rgroups = o.per_sample ? 1 : (l.R + kMaxRB - 1) / kMaxRB;
+            t.partial_base = slots;
+            t.seg_base = (int)ctx->segs.size();
+            t.amax_preset = o.amax_preset;
+            const long long my_tiles = o.per_sample ? (long long)l.R * t.tiles_per_seg
+                                                    : (long long)t.tiles_per_seg * t.rgroups;
+            const long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kTileElems - 1) / kTileElems;
+            ctx->tile_begin.push_back(tiles);
+            ctx->amax_tile_begin.push_back(atiles);
+            tiles += my_tiles;
+            atiles += my_atiles;
+            for (int r = 0; r < l.R; ++r) {
+                Segment s{};
+                s.first_slot = slots + (long long)r * t.tiles_per_seg;
+                s.count = t.tiles_per_seg;
+                ctx->segs.push_back(s);
+            }
+            slots += (long long)l.R * t.tiles_per_seg;
+            o.tensor = (int)ctx->tens.size();
+            if (k == 0) { ly.seg_base0 = t.seg_base; ly.tensor0 = o.tensor; }
+            else { ly.seg_base1 = t.seg_base; ly.tensor1 = o.tensor; }
+            ctx->tens.push_back(t);
+        }
+        l.scored = (int)ctx->lay.size();
+        ctx->lay.push_back(ly);
+        ctx->scored_layer_ids.push_back((int)li);
+    }
+    ctx->tile_begin.push_back(tiles);
+    ctx->amax_tile_begin.push_back(atiles);
+    ctx->ntiles = tiles;
+    ctx->namax_tiles = atiles;
+    ctx->nslots = slots;
+    ctx->layer_out_doubles = out_off;
+    if (tiles > 0x7FFFFFFFLL || atiles > 0x7FFFFFFFLL)
+        return fail(ctx, AMPQ_ERR_TOO_LARGE, "more than 2^31-1 tiles in one score");
+    return AMPQ_OK;
+}
+
+int upload_tables(ampq_ctx* ctx) {
+    const size_t T = ctx->tens.size(), L = ctx->lay.size(), S = ctx->segs.size();
+    const int nacc = 1 + (ctx->F - 1);
+    AMPQ_CUDA(ctx->d_tens.ensure(T), "cudaMalloc(tensors)");
+    AMPQ_CUDA(ctx->d_tile_begin.ensure(T + 1), "cudaMalloc(tile_begin)");
+    AMPQ_CUDA(ctx->d_amax_tile_begin.ensure(T + 1), "cudaMalloc(amax_tile_begin)");
+    AMPQ_CUDA(ctx->d_segs.ensure(S), "cudaMalloc(segments)");
+    AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
+    AMPQ_CUDA(ctx->d_amax_bits.ensure(T), "cudaMalloc(amax)");
+    AMPQ_CUDA(ctx->d_scales.ensure(T * 2 * kMaxLow), "cudaMalloc(scales)");
+    AMPQ_CUDA(ctx->d_flags.ensure(T), "cudaMalloc(flags)");
+    AMPQ_CUDA(ctx->d_partials.ensure((size_t)ctx->nslots * nacc), "cudaMalloc(partials)");
+    AMPQ_CUDA(ctx->d_seg_out.ensure(S * nacc), "cudaMalloc(seg_out)");
+    AMPQ_CUDA(ctx->d_layer_out.ensure((size_t)ctx->layer_out_doubles), "cudaMalloc(layer_out)");
+    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
+    AMPQ_CUDA(ctx->h_amax_bits.ensure(T), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_scales.ensure(T * 2 * kMaxLow), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_flags.ensure(T), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_seg_out.ensure(S * nacc), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_layer_out.ensure((size_t)ctx->layer_out_doubles), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_status.ensure(1), "cudaMallocHost");
+    cudaStream_t st = ctx->stream;
+    if (T) {
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tens.p, ctx->tens.data(), T * sizeof(Tensor), cudaMemcpyHostToDevice, st), "H2D tensors");
+        AMPQ_CUDA(cudaMemsetAsync(ctx->d_scales.p, 0, T * 2 * kMaxLow * sizeof(float), st), "memset scales");
+    }
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tile_begin.p, ctx->tile_begin.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D tile_begin");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->d_amax_tile_begin.p, ctx->amax_tile_begin.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D amax_tile_begin");
+    if (S) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_segs.p, ctx->segs.data(), S * sizeof(Segment), cudaMemcpyHostToDevice, st), "H2D segments");
+    if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
+    return AMPQ_OK;
+}
+
+// Copies host-bound operands into their device staging on the stream.
+int stage_host_operands(ampq_ctx* ctx) {
+    for (auto& l : ctx->layers) {
+        if (l.scored < 0) continue;
+        for (int k = 0; k < 2; ++k) {
+            Operand& o = l.op[k];
+            if (o.mem != AMPQ_MEM_HOST || o.numel == 0) continue;
+            const int es = o.dtype == AMPQ_F32 ? 4 : 2;
+            const long long ext = extent_of(l, o);
+            char* dst = reinterpret_cast<char*>(o.stage);
+            AMPQ_CUDA(cudaMemcpyAsync(dst, o.values, (size_t)o.numel * es, cudaMemcpyHostToDevice, ctx->stream), "H2D values");
+            dst += (((size_t)o.numel * es) + 255) / 256 * 256;
+            if (o.grad_stride == ext) {
+                AMPQ_CUDA(cudaMemcpyAsync(dst, o.grads, (size_t)l.R * ext * es, cudaMemcpyHostToDevice, ctx->stream), "H2D grads");
+            } else {
+                for (int r = 0; r < l.R; ++r)
+                    AMPQ_CUDA(cudaMemcpyAsync(dst + (size_t)r * ext * es,
+                                              reinterpret_cast<const char*>(o.grads) + (size_t)r * o.grad_stride * es,
+                                              (size_t)ext * es, cudaMemcpyHostToDevice, ctx->stream), "H2D grads");
+            }
+        }
+    }
+    return AMPQ_OK;
+}
+
+int sync_results(ampq_ctx* ctx) {
+    if (!ctx->scored) return fail(ctx, AMPQ_ERR_STATE, "no score has been issued");
+    if (ctx->pending) {
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        ctx->pending = false;
+    }
+    return AMPQ_OK;
+}
+
+int check_layer(ampq_ctx* ctx, int layer_id) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    if (layer_id < 0 || layer_id >= (int)ctx->layers.size()) return fail(ctx, AMPQ_ERR_INVALID, "unknown layer id");
+    return AMPQ_OK;
+}
+
+const double* layer_block(const ampq_ctx* ctx, int scored) {
+    return ctx->h_layer_out.p + ctx->lay[scored].out_off;
+}
+
+// d_{l,f} of a scored layer from the last score.
+double layer_d(const ampq_ctx* ctx, int scored, int f, int d_mode) {
+    const int R = ctx->lay[scored].R, F = ctx->F;
+    const double* o = layer_block(ctx, scored);
+    const double* d_model = o + R + 1 + (long long)R * F;
+    const double* d_meas = d_model + F;
+    return d_mode == AMPQ_D_MEASURED ? d_meas[f] : d_model[f];
+}
+
+int group_costs_impl(ampq_ctx* ctx, const Group& g, int d_mode, double* d_out) {
+    const int Lj = (int)g.layers.size();
+    for (int l = 0; l < Lj; ++l) {
+        if (ctx->layers[g.layers[l]].scored < 0)
+            return fail(ctx, AMPQ_ERR_STATE, "a layer of the group was not part of the last score");
+        const int sc = ctx->layers[g.layers[l]].scored;
+        if (ctx->h_flags.p[ctx->lay[sc].tensor0] || ctx->h_flags.p[ctx->lay[sc].tensor1])
+            return fail(ctx, AMPQ_ERR_NONFINITE, "layer '" + ctx->layers[g.layers[l]].name + "' holds Inf/NaN");
+    }
+    for (int p = 0; p < g.P; ++p) {
+        double d = 0.0;
+        for (int l = 0; l < Lj; ++l)
+            d += layer_d(ctx, ctx->layers[g.layers[l]].scored, g.Q[l + (size_t)Lj * p], d_mode);
+        d_out[p] = d;
+    }
+    return AMPQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char* ampq_strerror(int status) {
+    switch (status) {
+        case AMPQ_OK: return "ok";
+        case AMPQ_ERR_INVALID: return "invalid argument";
+        case AMPQ_ERR_ALIGN: return "tensor pointer not aligned to its element size";
+        case AMPQ_ERR_STATE: return "call out of order";
+        case AMPQ_ERR_CUDA: return "CUDA error";
+        case AMPQ_ERR_NONFINITE: return "operand holds Inf or NaN";
+        case AMPQ_ERR_INFEASIBLE: return "no assignment meets the budget";
+        case AMPQ_ERR_TOO_LARGE: return "problem too large";
+        case AMPQ_ERR_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+const char* ampq_last_error(const ampq_ctx* ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+int ampq_create(ampq_ctx** out, int device, void* cuda_stream) {
+    if (!out) return AMPQ_ERR_INVALID;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return AMPQ_ERR_CUDA; }
+    if (device < 0 || device >= n) return AMPQ_ERR_INVALID;
+    ampq_ctx* ctx = new (std::nothrow) ampq_ctx();
+    if (!ctx) return AMPQ_ERR_NOMEM;
+    ctx->device = device;
+    ctx->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard g(device);
+    if (!g.ok || cudaFree(nullptr) != cudaSuccess) { delete ctx; return AMPQ_ERR_CUDA; }
+    *out = ctx;
+    return AMPQ_OK;
+}
+
+int ampq_destroy(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_OK;
+    {
+        DeviceGuard g(ctx->device);
+        if (ctx->pending) cudaStreamSynchronize(ctx->stream);
+        for (auto& l : ctx->layers)
+            for (int k = 0; k < 2; ++k)
+                if (l.op[k].stage) cudaFree(l.op[k].stage);
+        ctx->d_tens.release(); ctx->d_tile_begin.release(); ctx->d_amax_tile_begin.release();
+        ctx->d_segs.release(); ctx->d_lay.release(); ctx->d_amax_bits.release(); ctx->d_scales.release();
+        ctx->d_partials.release(); ctx->d_flags.release(); ctx->d_seg_out.release();
+        ctx->d_layer_out.release(); ctx->d_status.release();
+        ctx->h_amax_bits.release(); ctx->h_scales.release(); ctx->h_flags.release();
+        ctx->h_seg_out.release(); ctx->h_layer_out.release(); ctx->h_status.release();
+    }
+    delete ctx;
+    return AMPQ_OK;
+}
+
+int ampq_set_formats(ampq_ctx* ctx, const int* fmt, int F) {
+    if (!ctx || !fmt) return AMPQ_ERR_INVALID;
+    if (F < 2 || F > 1 + kMaxLow) return fail(ctx, AMPQ_ERR_INVALID, "F must be 2 or 3");
+    if (fmt[0] != AMPQ_FMT_BASE) return fail(ctx, AMPQ_ERR_INVALID, "fmt[0] must be AMPQ_FMT_BASE");
+    int mask = 0;
+    for (int f = 1; f < F; ++f) {
+        if (fmt[f] != AMPQ_FMT_E4M3 && fmt[f] != AMPQ_FMT_E5M2) return fail(ctx, AMPQ_ERR_INVALID, "unknown low-precision format");
+        const int bit = fmt[f] == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2;
+        if (mask & bit) return fail(ctx, AMPQ_ERR_INVALID, "duplicate format");
+        mask |= bit;
+    }
+    ctx->F = F;
+    ctx->fmask = mask;
+    for (int f = 0; f < 1 + kMaxLow; ++f) { ctx->fmt[f] = f < F ? fmt[f] : 0; ctx->slot_of_fmt[f] = -1; }
+    for (int f = 1; f < F; ++f) ctx->slot_of_fmt[f] = (mask == 3 && fmt[f] == AMPQ_FMT_E5M2) ? 1 : 0;
+    ctx->dirty = true;
+    ctx->scored = false;
+    return AMPQ_OK;
+}
+
+int ampq_register_layer(ampq_ctx* ctx, int kind, const char* name, int R, int* layer_id) {
+    if (!ctx || !layer_id) return AMPQ_ERR_INVALID;
+    if (kind != AMPQ_LINEAR && kind != AMPQ_BGEMM) return fail(ctx, AMPQ_ERR_INVALID, "unknown layer kind");
+    if (R < 1) return fail(ctx, AMPQ_ERR_INVALID, "R must be at least 1");
+    LayerRec l;
+    l.kind = kind;
+    l.R = R;
+    if (name) l.name = name;
+    ctx->layers.push_back(l);
+    *layer_id = (int)ctx->layers.size() - 1;
+    return AMPQ_OK;
+}
+
+int ampq_bind_operand(ampq_ctx* ctx, int layer_id, int operand, int dtype, int mem, const void* values,
+                      long long numel, int per_sample_values, const void* grads, long long grad_stride) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
+    if (dtype != AMPQ_F32 && dtype != AMPQ_BF16) return fail(ctx, AMPQ_ERR_INVALID, "unknown dtype");
+    if (mem != AMPQ_MEM_DEVICE && mem != AMPQ_MEM_HOST) return fail(ctx, AMPQ_ERR_INVALID, "unknown memory kind");
+    if (numel < 0) return fail(ctx, AMPQ_ERR_INVALID, "negative numel");
+    LayerRec& l = ctx->layers[layer_id];
+    if (numel > 0 && (!values || !grads)) return fail(ctx, AMPQ_ERR_INVALID, "null tensor pointer");
+    if (per_sample_values && numel % l.R != 0) return fail(ctx, AMPQ_ERR_INVALID, "numel is not a multiple of R");
+    const long long ext = per_sample_values ? numel / l.R : numel;
+    if (l.R > 1 && grad_stride < ext) return fail(ctx, AMPQ_ERR_INVALID, "grad_stride is smaller than one sample's gradient");
+    const int es = dtype == AMPQ_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(values) % es) || (reinterpret_cast<uintptr_t>(grads) % es))
+        return fail(ctx, AMPQ_ERR_ALIGN, "tensor pointer not aligned to its element size");
+    Operand& o = l.op[operand];
+    o.bound = true;
+    o.dtype = dtype; o.mem = mem; o.per_sample = per_sample_values ? 1 : 0;
+    o.values = values; o.grads = grads; o.numel = numel; o.grad_stride = grad_stride;
+    ctx->dirty = true;
+    return AMPQ_OK;
+}
+
+int ampq_set_amax(ampq_ctx* ctx, int layer_id, int operand, float amax) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
+    if (amax != amax || std::isinf(amax)) return fail(ctx, AMPQ_ERR_INVALID, "amax must be finite");
+    ctx->layers[layer_id].op[operand].amax_preset = amax >= 0.0f ? amax : -1.0f;
+    ctx->dirty = true;
+    return AMPQ_OK;
+}
+
+int ampq_score(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    int rc;
+    if (ctx->pending) {  // the previous score's read-back still owns the pinned mirrors
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        ctx->pending = false;
+    }
+    if (ctx->dirty) {
+        ctx->scored = false;
+        if ((rc = build_tables(ctx))) return rc;
+        if ((rc = upload_tables(ctx))) return rc;
+        ctx->dirty = false;
+    }
+    const int T = (int)ctx->tens.size(), L = (int)ctx->lay.size(), S = (int)ctx->segs.size();
+    const int nacc = ctx->F;  // S plus one D per low-precision format
+    cudaStream_t st = ctx->stream;
+    ctx->launches = 0;
+    if ((rc = stage_host_operands(ctx))) return rc;
+    if (T > 0) {
+        AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
+        ++ctx->launches;
+        if (ctx->namax_tiles > 0) {
+            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
+            ++ctx->launches;
+        }
+        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st), "scales");
+        ++ctx->launches;
+        if (ctx->ntiles > 0) {
+            AMPQ_CUDA(launch_score(ctx->d_tens.p, ctx->d_tile_begin.p, T, ctx->ntiles, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, st), "score");
+            ++ctx->launches;
+        }
+        AMPQ_CUDA(launch_finalize(ctx->d_segs.p, S, nacc, ctx->d_partials.p, ctx->d_seg_out.p, st), "finalize");
+        ++ctx->launches;
+        CombineParams prm{};
+        prm.nacc = nacc;
+        for (int f = 1; f < ctx->F; ++f) {
+            prm.alpha[f] = std::ldexp(1.0, -2 * mantissa_bits_of(ctx->fmt[f])) / 12.0;
+            prm.acc_of_fmt[f] = 1 + ctx->slot_of_fmt[f];
+        }
+        AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, prm, ctx->d_seg_out.p, ctx->d_layer_out.p, st), "combine");
+        ++ctx->launches;
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_scales.p, ctx->d_scales.p, (size_t)T * 2 * kMaxLow * sizeof(float), cudaMemcpyDeviceToHost, st), "D2H scales");
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_flags.p, ctx->d_flags.p, T * sizeof(int), cudaMemcpyDeviceToHost, st), "D2H flags");
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_seg_out.p, ctx->d_seg_out.p, (size_t)S * nacc * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H segments");
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_layer_out.p, ctx->d_layer_out.p, (size_t)ctx->layer_out_doubles * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H layers");
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_status.p, ctx->d_status.p, sizeof(LaunchStatus), cudaMemcpyDeviceToHost, st), "D2H status");
+    }
+    ctx->scored = true;
+    ctx->pending = T > 0;
+    return AMPQ_OK;
+}
+
+int ampq_last_launch_count(const ampq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int ampq_get_layer(ampq_ctx* ctx, int layer_id, float* amax, float* scale, float* inv_scale,
+                   double* s_per_sample, double* s_mean, double* d_meas_per_sample, double* d_model,
+                   double* d_meas) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    DeviceGuard g(ctx->device);
+    if ((rc = sync_results(ctx))) return rc;
+    const LayerRec& l = ctx->layers[layer_id];
+    if (l.scored < 0) return fail(ctx, AMPQ_ERR_STATE, "layer was not part of the last score");
+    const Layer& ly = ctx->lay[l.scored];
+    const int F = ctx->F, R = ly.R;
+    const int tix[2] = {ly.tensor0, ly.tensor1};
+    bool bad = false;
+    for (int k = 0; k < 2; ++k) {
+        const int t = tix[k];
+        bad = bad || ctx->h_flags.p[t] != 0;
+        if (amax) std::memcpy(&amax[k], &ctx->h_amax_bits.p[t], sizeof(float));
+        for (int f = 0; f < F; ++f) {
+            float sc = 1.0f, iv = 1.0f;
+            if (f > 0) {
+                sc = ctx->h_scales.p[t * 2 * kMaxLow + ctx->slot_of_fmt[f] * 2 + 0];
+                iv = ctx->h_scales.p[t * 2 * kMaxLow + ctx->slot_of_fmt[f] * 2 + 1];
+            }
+            if (scale) scale[k * F + f] = sc;
+            if (inv_scale) inv_scale[k * F + f] = iv;
+        }
+    }
+    const double* o = layer_block(ctx, l.scored);
+    if (s_per_sample) std::memcpy(s_per_sample, o, sizeof(double) * R);
+    if (s_mean) *s_mean = o[R];
+    if (d_meas_per_sample) std::memcpy(d_meas_per_sample, o + R + 1, sizeof(double) * R * F);
+    if (d_model) std::memcpy(d_model, o + R + 1 + (long long)R * F, sizeof(double) * F);
+    if (d_meas) std::memcpy(d_meas, o + R + 1 + (long long)R * F + F, sizeof(double) * F);
+    if (bad) return fail(ctx, AMPQ_ERR_NONFINITE, "layer '" + l.name + "' holds Inf/NaN");
+    return AMPQ_OK;
+}
+
+int ampq_get_operand(ampq_ctx* ctx, int layer_id, int operand, double* out) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if ((operand != 0 && operand != 1) || !out) return fail(ctx, AMPQ_ERR_INVALID, "bad operand or null output");
+    DeviceGuard g(ctx->device);
+    if ((rc = sync_results(ctx))) return rc;
+    const LayerRec& l = ctx->layers[layer_id];
+    if (l.scored < 0) return fail(ctx, AMPQ_ERR_STATE, "layer was not part of the last score");
+    const Layer& ly = ctx->lay[l.scored];
+    const int F = ctx->F, nacc = F;
+    const int sb = operand == 0 ? ly.seg_base0 : ly.seg_base1;
+    for (int r = 0; r < ly.R; ++r) {
+        out[r * F] = ctx->h_seg_out.p[(size_t)(sb + r) * nacc];
+        for (int f = 1; f < F; ++f)
+            out[r * F + f] = ctx->h_seg_out.p[(size_t)(sb + r) * nacc + 1 + ctx->slot_of_fmt[f]];
+    }
+    return AMPQ_OK;
+}
+
+int ampq_export_codes(ampq_ctx* ctx, int layer_id, int operand, int fmt, unsigned char* dev_out) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
+    if (!ctx->scored || ctx->dirty) return fail(ctx, AMPQ_ERR_STATE, "export needs the scales of a score of the current bindings");
+    const LayerRec& l = ctx->layers[layer_id];
+    const Operand& o = l.op[operand];
+    if (l.scored < 0 || o.tensor < 0) return fail(ctx, AMPQ_ERR_STATE, "layer was not part of the last score");
+    if (o.mem != AMPQ_MEM_DEVICE) return fail(ctx, AMPQ_ERR_INVALID, "export needs a device-bound operand");
+    int f = -1;
+    for (int k = 1; k < ctx->F; ++k)
+        if (ctx->fmt[k] == fmt) f = k;
+    if (f < 0) return fail(ctx, AMPQ_ERR_INVALID, "format is not in the context's format list");
+    if (o.numel > 0 && !dev_out) return fail(ctx, AMPQ_ERR_INVALID, "null output");
+    DeviceGuard g(ctx->device);
+    const float* pair = ctx->d_scales.p + (size_t)o.tensor * 2 * kMaxLow + ctx->slot_of_fmt[f] * 2;
+    AMPQ_CUDA(launch_codes(o.dtype, fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2, o.values, o.numel, pair, dev_out, ctx->stream), "codes");
+    return AMPQ_OK;
+}
+
+int ampq_define_group(ampq_ctx* ctx, const int* layer_ids, int Lj, const unsigned char* Q, const double* c,
+                      int Pj, int* group_id) {
+    if (!ctx || !layer_ids || !Q || !c || !group_id) return AMPQ_ERR_INVALID;
+    if (Lj < 1 || Pj < 1) return fail(ctx, AMPQ_ERR_INVALID, "a group needs at least one layer and one configuration");
+    Group g;
+    for (int l = 0; l < Lj; ++l) {
+        if (layer_ids[l] < 0 || layer_ids[l] >= (int)ctx->layers.size()) return fail(ctx, AMPQ_ERR_INVALID, "unknown layer id in group");
+        g.layers.push_back(layer_ids[l]);
+    }
+    for (long long i = 0; i < (long long)Lj * Pj; ++i)
+        if (Q[i] >= ctx->F) return fail(ctx, AMPQ_ERR_INVALID, "Q entry outside the format list");
+    for (int p = 0; p < Pj; ++p)
+        if (c[p] != c[p]) return fail(ctx, AMPQ_ERR_INVALID, "metric is NaN");
+    g.Q.assign(Q, Q + (size_t)Lj * Pj);
+    g.c.assign(c, c + Pj);
+    g.P = Pj;
+    ctx->groups.push_back(std::move(g));
+    *group_id = (int)ctx->groups.size() - 1;
+    return AMPQ_OK;
+}
+
+int ampq_clear_groups(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    ctx->groups.clear();
+    return AMPQ_OK;
+}
+
+int ampq_group_costs(ampq_ctx* ctx, int group_id, int d_mode, double* d_out) {
+    if (!ctx || !d_out) return AMPQ_ERR_INVALID;
+    if (group_id < 0 || group_id >= (int)ctx->groups.size()) return fail(ctx, AMPQ_ERR_INVALID, "unknown group id");
+    if (d_mode != AMPQ_D_MODEL && d_mode != AMPQ_D_MEASURED) return fail(ctx, AMPQ_ERR_INVALID, "unknown d_mode");
+    DeviceGuard g(ctx->device);
+    int rc = sync_results(ctx);
+    if (rc) return rc;
+    return group_costs_impl(ctx, ctx->groups[group_id], d_mode, d_out);
+}
+
+int ampq_budget_from_tau(double tau, const double* losses, int R, double* budget) {
+    if (!losses || !budget || R < 1 || !(tau >= 0.0)) return AMPQ_ERR_INVALID;
+    double a = 0.0;
+    for (int r = 0; r < R; ++r) a += losses[r] * losses[r];
+    *budget = tau * tau * (a / (double)R);
+    return AMPQ_OK;
+}
+
+int ampq_all_lowp_cost(ampq_ctx* ctx, int d_mode, int f, double* d_all) {
+    if (!ctx || !d_all) return AMPQ_ERR_INVALID;
+    if (f < 1 || f >= ctx->F) return fail(ctx, AMPQ_ERR_INVALID, "format index must be 1..F-1");
+    if (d_mode != AMPQ_D_MODEL && d_mode != AMPQ_D_MEASURED) return fail(ctx, AMPQ_ERR_INVALID, "unknown d_mode");
+    DeviceGuard g(ctx->device);
+    int rc = sync_results(ctx);
+    if (rc) return rc;
+    double d = 0.0;
+    for (size_t s = 0; s < ctx->lay.size(); ++s) {
+        if (ctx->h_flags.p[ctx->lay[s].tensor0] || ctx->h_flags.p[ctx->lay[s].tensor1])
+            return fail(ctx, AMPQ_ERR_NONFINITE, "a scored layer holds Inf/NaN");
+        d += layer_d(ctx, (int)s, f, d_mode);
+    }
+    *d_all = d;
+    return AMPQ_OK;
+}
+
+int ampq_select_tables(int J, const int* P, const long long* off, const double* c, const double* d,
+                       double budget, int* p_out, double* c_total, double* d_total) {
+    if (J < 0 || (J > 0 && (!P || !off || !c || !d || !p_out))) return AMPQ_ERR_INVALID;
+    const int rc = select_mckp(J, P, off, c, d, budget, 50000000LL, p_out, c_total, d_total);
+    switch (rc) {
+        case kSelectOk: return AMPQ_OK;
+        case kSelectInfeasible: return AMPQ_ERR_INFEASIBLE;
+        case kSelectTooLarge: return AMPQ_ERR_TOO_LARGE;
+        default: return AMPQ_ERR_INVALID;
+    }
+}
+
+int ampq_select(ampq_ctx* ctx, int d_mode, double budget, int* p_out, double* c_total, double* d_total) {
+    if (!ctx || !p_out) return AMPQ_ERR_INVALID;
+    if (d_mode != AMPQ_D_MODEL && d_mode != AMPQ_D_MEASURED) return fail(ctx, AMPQ_ERR_INVALID, "unknown d_mode");
+    DeviceGuard g(ctx->device);
+    int rc = sync_results(ctx);
+    if (rc) return rc;
+    const int J = (int)ctx->groups.size();
+    std::vector<int> P(J);
+    std::vector<long long> off(J);
+    std::vector<double> c, d;
+    for (int j = 0; j < J; ++j) {
+        const Group& gr = ctx->groups[j];
+        P[j] = gr.P;
+        off[j] = (long long)c.size();
+        c.insert(c.end(), gr.c.begin(), gr.c.end());
+        d.resize(d.size() + gr.P);
+        if ((rc = group_costs_impl(ctx, gr, d_mode, d.data() + off[j]))) return rc;
+    }
+    rc = ampq_select_tables(J, P.data(), off.data(), c.data(), d.data(), budget, p_out, c_total, d_total);
+    if (rc == AMPQ_ERR_INFEASIBLE) ctx->err = "no assignment meets the budget";
+    if (rc == AMPQ_ERR_TOO_LARGE) ctx->err = "selection exceeded its state limit";
+    return rc;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -35,3 +35,14 @@ def read_golden(name):
             k, v = line.split("=", 1)
             out[k.strip()] = v.strip()
     return out
+
+
+@pytest.fixture(scope="session")
+def ampq():
+    """The ctypes binding of the CUDA library (built with nvcc when stale)."""
+    from paper_2505_13060_b200 import binding, build
+
+    if build.needs_build():
+        build.build()
+    binding.lib()
+    return binding

@@ -1,0 +1,340 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element on
+the same seeded tensors, through the C ABI.  Run with -m gpu on a B200."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, compare_layer, gpu_codes, oracle_layer
+from paper_2505_13060_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+E4M3, E5M2 = 1, 2
+
+
+def _ctx(ampq, fmts=(0, E4M3)):
+    ctx = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
+    ctx.set_formats(list(fmts))
+    return ctx
+
+
+def _register(ampq, ctx, lts):
+    ids = []
+    for lt in lts:
+        lid = ctx.register_layer(lt.spec.kind, lt.spec.name, lt.spec.R)
+        ampq.bind_layer_tensors(ctx, lid, lt)
+        ids.append(lid)
+    return ids
+
+
+def _mac_gain_groups(ctx, ids, specs, group_size):
+    """Groups of consecutive layers with every format combination as a column
+    and the MAC count of the low-precision layers as the metric."""
+    tabs = []
+    for g0 in range(0, len(ids), group_size):
+        members = list(range(g0, min(g0 + group_size, len(ids))))
+        Lj = len(members)
+        P = 2 ** Lj
+        Q = np.array([[(p >> l) & 1 for p in range(P)] for l in range(Lj)], dtype=np.uint8)
+        c = np.array([sum(specs[m].mac for l, m in enumerate(members) if (p >> l) & 1) for p in range(P)], float)
+        ctx.define_group([ids[m] for m in members], Q, c)
+        tabs.append((members, Q, c))
+    return tabs
+
+
+@pytest.mark.parametrize("fmts", [(0, E4M3), (0, E5M2), (0, E4M3, E5M2), (0, E5M2, E4M3)])
+def test_toy_mlp_whole(ampq, orc, fmts):
+    """The toy MLP (4 fp32 linear layers, R = 8): every value the library returns."""
+    specs = synth.toy_mlp()
+    lts = [synth.make_layer(s, "cuda", seed=0, layer=i) for i, s in enumerate(specs)]
+    ctx = _ctx(ampq, fmts)
+    ids = _register(ampq, ctx, lts)
+    ctx.score()
+    low = list(fmts[1:])
+    refs = [oracle_layer(orc, lt, low) for lt in lts]
+    for lid, lt, ref in zip(ids, lts, refs):
+        compare_layer(ampq, ctx, lid, ref, len(fmts), lt.spec.name)
+        for k in range(2):
+            for fi, f in enumerate(low):
+                want = orc.codes(synth.to_numpy(lt.values[k]), f, ref["ops"][k]["inv"][fi])
+                got = gpu_codes(ctx, lid, k, f, lt.values[k].numel())
+                assert np.array_equal(got, want), (lt.spec.name, k, f)
+    # the measured term sits where the noise model says it should (Sec. 2.2)
+    for ref in refs:
+        for f in range(1, len(fmts)):
+            assert 0.2 * ref["d_model"][f] < ref["d_meas"][f] < 1.2 * ref["d_model"][f]
+    # two sub-graphs of two layers, all four columns, budget = half the all-FP8 loss MSE
+    tabs = _mac_gain_groups(ctx, ids, specs, 2)
+    for mode, key in ((ampq.D_MODEL, "d_model"), (ampq.D_MEASURED, "d_meas")):
+        d_layer = np.array([r[key] for r in refs])
+        d_tabs = [orc.group_costs(m, Q, d_layer) for m, Q, _ in tabs]
+        for j, dt in enumerate(d_tabs):
+            assert_close(ctx.group_costs(j, mode), dt, "group %d costs" % j)
+        all_low = float(np.sum(d_layer[:, 1]))
+        assert_close(ctx.all_lowp_cost(mode, 1), all_low, "all-low-precision cost")
+        for frac in (0.0, 0.25, 0.5, 0.75, 1.0001):
+            want = orc.select_bruteforce([c for _, _, c in tabs], d_tabs, frac * all_low)
+            got = ctx.select(mode, frac * ctx.all_lowp_cost(mode, 1))
+            assert got[0].tolist() == want[0].tolist(), (mode, frac)
+            assert got[1] == want[1]
+            assert_close(got[2], want[2], "selected d") if want[2] else None
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("R", [1, 2, 3, 5, 8])
+def test_ragged_sizes_and_sample_groups(ampq, orc, dtype, R):
+    """Sizes that are not multiples of a vector or a tile, segments that start
+    off 16-byte boundaries, and every split of R into shared-value groups."""
+    ctx = _ctx(ampq, (0, E4M3, E5M2))
+    lts = []
+    for li, (nx, nw) in enumerate([(1, 7), (9, 32768), (32769, 65537), (40003, 3), (70001, 100000)]):
+        spec = synth.LayerSpec("rag%d" % li, synth.LINEAR, R, dtype,
+                               synth.OperandSpec((R, nx), True, 1.0, 1e-3),
+                               synth.OperandSpec((nw,), False, 0.02, 1e-3))
+        lts.append(synth.make_layer(spec, "cuda", seed=3, layer=li))
+    ids = _register(ampq, ctx, lts)
+    ctx.score()
+    for lid, lt in zip(ids, lts):
+        compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, [E4M3, E5M2]), 3, lt.spec.name)
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_misaligned_pointers_and_strides(ampq, orc, dtype):
+    """Tensors that start one element past a 16-byte boundary, and gradients
+    whose sample stride is larger than one sample."""
+    R, n = 3, 50001
+    es = torch.empty((), dtype=dtype).element_size()
+    g = torch.Generator(device="cuda").manual_seed(5)
+    buf_v = torch.empty(R * n + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g)
+    stride = n + 13
+    buf_g = (torch.empty(R * stride + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g) * 1e-3)
+    w = torch.empty(n + 16, dtype=dtype, device="cuda").normal_(0, 0.02, generator=g)
+    gw = (torch.empty(R * stride + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g) * 1e-3)
+    ctx = _ctx(ampq)
+    lid = ctx.register_layer(ampq.LINEAR, "mis", R)
+    code = ampq.torch_dtype_code(buf_v)
+    ctx.bind_operand(lid, 0, code, buf_v.data_ptr() + es, R * n, True, buf_g.data_ptr() + es, stride)
+    ctx.bind_operand(lid, 1, code, w.data_ptr() + 3 * es, n, False, gw.data_ptr() + es, stride)
+    ctx.score()
+
+    class LT:  # the same views for the oracle
+        pass
+
+    lt = LT()
+    lt.spec = synth.LayerSpec("mis", synth.LINEAR, R, dtype, synth.OperandSpec((R, n), True),
+                              synth.OperandSpec((n,), False))
+    lt.values = [buf_v[1:1 + R * n].reshape(R, n), w[3:3 + n]]
+    lt.grads = [torch.stack([buf_g[1 + r * stride: 1 + r * stride + n] for r in range(R)]),
+                torch.stack([gw[1 + r * stride: 1 + r * stride + n] for r in range(R)])]
+    compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, [E4M3]), 2, "misaligned")
+    # an odd byte address is refused
+    assert ampq.lib().ampq_bind_operand(ctx._h, lid, 0, code, 0, buf_v.data_ptr() + 1, 9, 1,
+                                        buf_g.data_ptr(), 9) == ampq.ERR_ALIGN
+    ctx.destroy()
+
+
+def test_exhaustive_bf16_cast(ampq, orc):
+    """Every finite bf16 bit pattern through the cast, at several scales:
+    the exported codes must equal the oracle's bit for bit."""
+    pats = torch.arange(65536, dtype=torch.int32)
+    finite = (pats & 0x7F80) != 0x7F80
+    pats = pats[finite].to(torch.int16)
+    vals = pats.view(torch.bfloat16).cuda().contiguous()
+    n = vals.numel()
+    grads = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    host = synth.to_numpy(vals)
+    rng = np.random.default_rng(0)
+    amaxes = [448.0, 57344.0, 1.0, 2.0 ** -20, 2.0 ** 30, 3.3895e38] + list(np.exp(rng.uniform(-30, 30, 6)))
+    for a in amaxes:
+        ctx = _ctx(ampq, (0, E4M3, E5M2))
+        lid = ctx.register_layer(ampq.LINEAR, "cast", 1)
+        for k in range(2):
+            ctx.bind_operand(lid, k, ampq.BF16, vals.data_ptr(), n, False, grads.data_ptr(), n)
+            ctx.set_amax(lid, k, float(np.float32(a)))
+        ctx.score()
+        got = ctx.get_layer(lid)
+        for fi, f in enumerate((E4M3, E5M2)):
+            sc, iv = orc.scales(f, np.float32(a))
+            assert got["scale"][0, 1 + fi] == sc and got["inv_scale"][0, 1 + fi] == iv
+            assert np.array_equal(gpu_codes(ctx, lid, 0, f, n), orc.codes(host, f, iv)), (a, f)
+        ctx.destroy()
+
+
+def test_fp32_cast_patterns(ampq, orc):
+    """fp32: every exponent with dense mantissa coverage around the rounding
+    boundaries, plus random bit patterns (finite only)."""
+    rng = np.random.default_rng(1)
+    exps = np.arange(0, 255, dtype=np.uint32)
+    mant_hi = np.arange(0, 64, dtype=np.uint32) << 17           # the bits the FP8 mantissa keeps, and two below
+    mant_lo = np.array([0, 1, 0xFFFF, 0x10000, 0x10001, 0x1FFFF], dtype=np.uint32)
+    m = (mant_hi[:, None] | mant_lo[None, :]).reshape(-1)
+    bits = ((exps[:, None] << 23) | m[None, :]).reshape(-1)
+    bits = np.concatenate([bits, bits | 0x80000000, rng.integers(0, 2 ** 32, 1 << 22, dtype=np.uint64).astype(np.uint32)])
+    bits = bits[(bits & 0x7F800000) != 0x7F800000]
+    host = bits.view(np.float32)
+    vals = torch.from_numpy(host.copy()).cuda()
+    n = vals.numel()
+    grads = torch.zeros(n, dtype=torch.float32, device="cuda")
+    for a in (448.0, 1.0, 12345.678, 1e-30, 1e30):
+        ctx = _ctx(ampq, (0, E4M3, E5M2))
+        lid = ctx.register_layer(ampq.LINEAR, "cast32", 1)
+        for k in range(2):
+            ctx.bind_operand(lid, k, ampq.F32, vals.data_ptr(), n, False, grads.data_ptr(), n)
+            ctx.set_amax(lid, k, a)
+        ctx.score()
+        for f in (E4M3, E5M2):
+            _, iv = orc.scales(f, np.float32(a))
+            assert np.array_equal(gpu_codes(ctx, lid, 0, f, n), orc.codes(host, f, iv)), (a, f)
+        ctx.destroy()
+
+
+@pytest.mark.parametrize("recipe", ["llama7b", "llama70b", "attention"])
+def test_llm_shaped_blocks_scaled_down(ampq, orc, recipe):
+    """One block of each LLM-shaped workload with its large dimensions divided
+    by 8 (several tiles per segment, ragged tails), every layer compared."""
+    specs = {"llama7b": lambda: synth.llama7b_block(8), "llama70b": lambda: synth.llama70b_block(8),
+             "attention": lambda: synth.attention_bgemm(8)}[recipe]()
+    lts = [synth.make_layer(s, "cuda", seed=1, layer=i) for i, s in enumerate(specs)]
+    ctx = _ctx(ampq, (0, E4M3, E5M2))
+    ids = _register(ampq, ctx, lts)
+    ctx.score()
+    refs = []
+    for lid, lt in zip(ids, lts):
+        ref = oracle_layer(orc, lt, [E4M3, E5M2], threads=8)
+        refs.append(ref)
+        compare_layer(ampq, ctx, lid, ref, 3, lt.spec.name)
+    if recipe == "attention":
+        # the causal softmax operand is full of exact zeros and values that land
+        # in the FP8 subnormal range; its codes must still match
+        lt = lts[1]
+        want = orc.codes(synth.to_numpy(lt.values[0]), E4M3, refs[1]["ops"][0]["inv"][0])
+        assert np.array_equal(gpu_codes(ctx, ids[1], 0, E4M3, lt.values[0].numel()), want)
+        assert (want == 0).mean() > 0.4
+    ctx.destroy()
+
+
+def test_selection_sweep_from_gpu_tables(ampq, orc):
+    """Budgets of 1/5/20/50 % of the all-low-precision loss MSE over many
+    single- and multi-layer groups with random time gains: the plan picked from
+    the GPU tables equals the plan the oracle picks from its own tables."""
+    specs = []
+    for b in range(4):
+        specs += synth.llama7b_block(32, prefix="b%d." % b)
+    lts = [synth.make_layer(s, "cuda", seed=2, layer=i) for i, s in enumerate(specs)]
+    rng = np.random.default_rng(0)
+    for fmt in (E4M3, E5M2):
+        ctx = _ctx(ampq, (0, fmt))
+        ids = _register(ampq, ctx, lts)
+        ctx.score()
+        refs = [oracle_layer(orc, lt, [fmt], threads=8) for lt in lts]
+        tabs = []
+        for b in range(4):  # per block: the attention linears and the MLP linears
+            for members in (list(range(7 * b, 7 * b + 4)), list(range(7 * b + 4, 7 * b + 7))):
+                Q = np.array([[0, 1]] * len(members), dtype=np.uint8)
+                c = np.array([0.0, rng.uniform(0.5, 2.0)])
+                ctx.define_group([ids[m] for m in members], Q, c)
+                tabs.append((members, Q, c))
+        for mode, key in ((ampq.D_MODEL, "d_model"), (ampq.D_MEASURED, "d_meas")):
+            d_layer = np.array([r[key] for r in refs])
+            d_tabs = [orc.group_costs(m, Q, d_layer) for m, Q, _ in tabs]
+            all_low = float(np.sum(d_layer[:, 1]))
+            for frac in (0.01, 0.05, 0.2, 0.5):
+                want = orc.select_bruteforce([c for _, _, c in tabs], d_tabs, frac * all_low)
+                got = ctx.select(mode, frac * ctx.all_lowp_cost(mode, 1))
+                assert got[0].tolist() == want[0].tolist(), (fmt, mode, frac)
+        ctx.destroy()
+
+
+def test_preset_amax_saturates(ampq, orc):
+    spec = synth.toy_mlp(R=2, tokens=64, width=128, layers=1)[0]
+    lt = synth.make_layer(spec, "cuda", seed=4)
+    ctx = _ctx(ampq)
+    (lid,) = _register(ampq, ctx, [lt])
+    ctx.set_amax(lid, 0, 2.5)   # well below the outliers: they saturate at +-448 * scale
+    ctx.score()
+    ref = oracle_layer(orc, lt, [E4M3], amax_presets=(2.5, None))
+    got = compare_layer(ampq, ctx, lid, ref, 2, "preset")
+    assert got["amax"][0] == np.float32(2.5)
+    codes = gpu_codes(ctx, lid, 0, E4M3, lt.values[0].numel())
+    assert (codes & 0x7F).max() == 0x7E
+    ctx.set_amax(lid, 0, -1.0)  # back to the measured amax
+    ctx.score()
+    compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, [E4M3]), 2, "measured again")
+    ctx.destroy()
+
+
+def test_degenerate_inputs(ampq, orc):
+    """Empty operands, all-zero tensors (amax = 0 -> scale 1), unbound layers,
+    non-finite values reported as an error code, calls out of order."""
+    ctx = _ctx(ampq)
+    z = torch.zeros(1000, dtype=torch.float32, device="cuda")
+    g = torch.ones(2000, dtype=torch.float32, device="cuda")
+    l0 = ctx.register_layer(ampq.LINEAR, "zeros", 2)
+    assert ampq.lib().ampq_get_layer(ctx._h, l0, *([None] * 8)) == ampq.ERR_STATE   # nothing scored yet
+    ctx.bind_operand(l0, 0, ampq.F32, z.data_ptr(), 1000, True, g.data_ptr(), 500)
+    ctx.bind_operand(l0, 1, ampq.F32, 0, 0, False, 0, 0)                              # empty operand
+    l1 = ctx.register_layer(ampq.BGEMM, "half-bound", 1)
+    ctx.bind_operand(l1, 0, ampq.F32, z.data_ptr(), 10, True, g.data_ptr(), 10)
+    bad = torch.randn(5000, device="cuda")
+    bad[4321] = float("inf")
+    l2 = ctx.register_layer(ampq.LINEAR, "nonfinite", 1)
+    ctx.bind_operand(l2, 0, ampq.F32, bad.data_ptr(), 5000, True, g.data_ptr(), 5000)
+    ctx.bind_operand(l2, 1, ampq.F32, z.data_ptr(), 100, False, g.data_ptr(), 100)
+    ctx.score()
+    r0 = ctx.get_layer(l0)
+    assert r0["amax"].tolist() == [0.0, 0.0] and r0["scale"][0, 1] == 1.0 and r0["s_mean"] == 0.0
+    assert r0["d_meas"].tolist() == [0.0, 0.0]
+    assert ampq.lib().ampq_get_layer(ctx._h, l1, *([None] * 8)) == ampq.ERR_STATE   # not scored
+    assert ctx.get_layer(l2, allow_nonfinite=True)["status"] == ampq.ERR_NONFINITE
+    gid = ctx.define_group([l2], np.array([[0, 1]], np.uint8), [0.0, 1.0])
+    with pytest.raises(ampq.AmpqError):
+        ctx.group_costs(gid)
+    L = ampq.lib()
+    assert L.ampq_bind_operand(ctx._h, 99, 0, 0, 0, None, 0, 0, None, 0) == ampq.ERR_INVALID
+    assert L.ampq_bind_operand(ctx._h, l0, 2, 0, 0, None, 0, 0, None, 0) == ampq.ERR_INVALID
+    assert L.ampq_bind_operand(ctx._h, l0, 0, 0, 0, z.data_ptr(), 999, 1, g.data_ptr(), 500) == ampq.ERR_INVALID
+    assert L.ampq_set_amax(ctx._h, l0, 0, float("nan")) == ampq.ERR_INVALID
+    with pytest.raises(ampq.AmpqError):
+        ctx.set_formats([1, 0])
+    ctx.destroy()
+
+
+def test_host_bound_operands_and_determinism(ampq, orc):
+    """Host-memory binding (staged by the library) gives exactly the device
+    result, and two scores of the same data are bit-identical."""
+    specs = synth.llama70b_block(16)[:3]
+    dev = [synth.make_layer(s, "cuda", seed=6, layer=i) for i, s in enumerate(specs)]
+    ctx = _ctx(ampq, (0, E4M3, E5M2))
+    ids = _register(ampq, ctx, dev)
+    ctx.score()
+    first = [(ctx.get_layer(i), ctx.get_operand(i, 0), ctx.get_operand(i, 1)) for i in ids]
+    ctx.score()
+    for i, (a, o0, o1) in zip(ids, first):
+        b = ctx.get_layer(i)
+        assert a["s_per_sample"].tobytes() == b["s_per_sample"].tobytes()
+        assert a["d_meas_per_sample"].tobytes() == b["d_meas_per_sample"].tobytes()
+        assert o0.tobytes() == ctx.get_operand(i, 0).tobytes() and o1.tobytes() == ctx.get_operand(i, 1).tobytes()
+    hctx = _ctx(ampq, (0, E4M3, E5M2))
+    keep = []
+    for lt in dev:
+        lid = hctx.register_layer(lt.spec.kind, lt.spec.name, lt.spec.R)
+
+        class H:
+            pass
+
+        h = H()
+        h.spec = lt.spec
+        h.values = [t.cpu().pin_memory() for t in lt.values]
+        h.grads = [t.cpu().pin_memory() for t in lt.grads]
+        keep.append(h)
+        ampq.bind_layer_tensors(hctx, lid, h, mem=ampq.MEM_HOST)
+    hctx.score()
+    for i, (a, o0, o1) in zip(ids, first):
+        b = hctx.get_layer(i)
+        assert a["amax"].tobytes() == b["amax"].tobytes()
+        assert a["s_per_sample"].tobytes() == b["s_per_sample"].tobytes()
+        assert a["d_meas"].tobytes() == b["d_meas"].tobytes()
+    hctx.destroy()
+    ctx.destroy()

@@ -1,0 +1,117 @@
+"""Host-side checks of the C-ABI library that need no GPU: the shared object
+loads and exports every symbol the header declares, argument errors are
+reported as status codes, and the exact selection agrees with the oracle's
+enumeration and branch and bound."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ampq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ampq_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(ampq):
+    names = _declared_symbols()
+    assert len(names) >= 20 and set(names) == set(ampq.EXPORTS)
+    L = ampq.lib()
+    for n in names:
+        assert getattr(L, n) is not None, n
+
+
+def test_status_strings_and_contextless_calls(ampq):
+    L = ampq.lib()
+    assert L.ampq_strerror(0) == b"ok"
+    for code in range(-8, 0):
+        assert L.ampq_strerror(code) not in (b"ok", b"unknown status")
+    assert ampq.budget_from_tau(0.1, [1.0, 2.0, 3.0]) == pytest.approx(0.01 * 14 / 3, rel=1e-15)
+    with pytest.raises(ampq.AmpqError):
+        ampq.budget_from_tau(-1.0, [1.0])
+    assert L.ampq_destroy(None) == 0
+    assert L.ampq_score(None) == ampq.ERR_INVALID
+
+
+def _rand_tables(rng, J, Pmax, integer=False):
+    c_tabs, d_tabs = [], []
+    for _ in range(J):
+        P = int(rng.integers(1, Pmax + 1))
+        if integer:
+            c = rng.integers(0, 4, P).astype(float)
+            d = rng.integers(0, 4, P).astype(float)
+        else:
+            c = rng.uniform(0, 2, P)
+            d = rng.uniform(0, 1, P) ** 3
+        if rng.random() < 0.7:
+            c[0], d[0] = 0.0, 0.0
+        c_tabs.append(c)
+        d_tabs.append(d)
+    return c_tabs, d_tabs
+
+
+@pytest.mark.parametrize("integer", [False, True])
+def test_select_matches_enumeration(ampq, orc, integer):
+    rng = np.random.default_rng(40 + integer)
+    for it in range(150):
+        c, d = _rand_tables(rng, int(rng.integers(1, 9)), 5, integer)
+        hi = sum(max(t) for t in d)
+        for budget in (0.0, 0.05 * hi, 0.3 * hi, 0.7 * hi, hi, 2 * hi + 1):
+            ref = orc.select_bruteforce(c, d, budget)
+            got = ampq.select_tables(c, d, budget)
+            if ref is None:
+                assert got is None
+                continue
+            assert got[0].tolist() == ref[0].tolist() and got[1] == ref[1] and got[2] == ref[2], (it, budget)
+
+
+def test_select_absorbing_magnitudes(ampq, orc):
+    """Terms spread over 18 orders of magnitude: partial sums absorb small
+    terms, so dominated prefixes can tie after rounding; the result must still
+    be the enumeration's."""
+    rng = np.random.default_rng(42)
+    for _ in range(20):
+        J = 12
+        c = [np.array([0.0, float(x)]) for x in 10.0 ** rng.uniform(-17, 1, J)]
+        d = [np.array([0.0, float(x)]) for x in 10.0 ** rng.uniform(-18, 0, J)]
+        hi = sum(t[1] for t in d)
+        for frac in (1e-6, 0.01, 0.3, 1.0):
+            ref = orc.select_bruteforce(c, d, frac * hi)
+            got = ampq.select_tables(c, d, frac * hi)
+            assert got[0].tolist() == ref[0].tolist() and got[1:] == ref[1:]
+
+
+@pytest.mark.parametrize("J,P", [(64, 2), (80, 2), (32, 16)])
+def test_select_large_matches_branch_and_bound(ampq, orc, J, P):
+    rng = np.random.default_rng(43)
+    c = [np.concatenate([[0.0], np.sort(rng.uniform(0.5, 2.0, P - 1))]) for _ in range(J)]
+    d = [np.concatenate([[0.0], np.sort(rng.uniform(0, 1, P - 1) ** 2)]) for _ in range(J)]
+    hi = sum(t[-1] for t in d)
+    prev = -1.0
+    for frac in (0.01, 0.05, 0.2, 0.5):
+        ref = orc.select_bnb(c, d, frac * hi, 50_000_000)
+        got = ampq.select_tables(c, d, frac * hi)
+        assert got[0].tolist() == ref[0].tolist() and got[1] == ref[1] and got[2] == ref[2]
+        assert got[2] <= frac * hi and got[1] >= prev
+        prev = got[1]
+
+
+def test_select_edge_cases(ampq):
+    assert ampq.select_tables([[1.0]], [[2.0]], 1.0) is None
+    p, c, d = ampq.select_tables([], [], 0.0)
+    assert len(p) == 0 and c == 0.0 and d == 0.0
+    with pytest.raises(ampq.AmpqError):
+        ampq.select_tables([[1.0]], [[-1.0]], 1.0)       # negative loss MSE
+    with pytest.raises(ampq.AmpqError):
+        ampq.select_tables([[float("nan")]], [[0.0]], 1.0)
+    # invariance to scale and bias of the metric
+    rng = np.random.default_rng(44)
+    c, d = _rand_tables(rng, 10, 4)
+    hi = sum(max(t) for t in d)
+    a = ampq.select_tables(c, d, 0.4 * hi)
+    b = ampq.select_tables([2.5 * t + 1.0 for t in c], d, 0.4 * hi)
+    assert a[0].tolist() == b[0].tolist()
