@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the loss-MSE sensitivity pass: GB/s scored on the Llama-70B-shaped workload.
+
+One step = one ``ampq_score`` over all 80 blocks x 7 linear layers of the
+70B-shaped configuration (hidden 8192, KV 1024, FFN 28672, R = 2 samples of 4096
+tokens, bf16): amax pass, scales, the fused FP8 cast / error / gradient
+weighting / reduction, ordered finalize and the per-layer combine, for
+614.7 GB of scored operand and gradient bytes.  80 blocks do not fit in HBM at
+once, so block b is bound to device slot b mod ``--resident-blocks`` (each slot
+is a full block of distinct random tensors, 7.68 GB); two passes over a slot are
+tens of GB of other traffic apart, far beyond the 126 MB L2, so every byte
+comes from HBM.
+
+Prints one JSON line: ``value`` = scored bytes of all ranks / device time of the
+step (CUDA events, max over ranks); ``roofline`` for the scoring kernel from
+events the library records around that kernel; ``e2e`` through the same C-ABI
+call with the tensors in pinned host memory (one block per step, copies inside
+the timed region); ``cpu_baseline`` = the CPU oracle timed on a bounded sample
+of the same workload.  ``--impl reference`` times only the oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sensitivity_pass_throughput_scored"
+UNIT = "GB/s"
+NUM_BLOCKS = 80
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--resident-blocks", type=int, default=8,
+                    help="distinct 70B-shaped blocks held on the device (7.68 GB each)")
+    ap.add_argument("--blocks", type=int, default=NUM_BLOCKS, help="blocks scored per step (the config has 80)")
+    ap.add_argument("--formats", default="e4m3", choices=["e4m3", "e5m2", "both"])
+    ap.add_argument("--workload", default="llama70b", choices=["llama70b", "llama7b"],
+                    help="llama70b is the benchmark; llama7b (3.2 GB per block) is the small case for profiler captures")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-threads", type=int, default=0)
+    return ap.parse_args()
+
+
+def hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------
+# clocks: nvidia-smi sampled while the timed region runs
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+                power.append(float(c[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# --------------------------------------------------------------------------
+def oracle_sample(threads: int, low_fmts, device):
+    """The oracle's bounded sample: the q, k, v, o linear layers of one
+    70B-shaped block (all R = 2 samples; 2.28 GB of scored bytes).  Returns
+    (host tensors per layer, scored bytes, description)."""
+    from paper_2505_13060_b200 import synth
+
+    specs = synth.llama70b_block()[:4]
+    layers, nbytes = [], 0
+    for i, s in enumerate(specs):
+        lt = synth.make_layer(s, device, seed=1234, layer=i)
+        layers.append((s, [synth.to_numpy(t) for t in lt.values], [synth.to_numpy(t) for t in lt.grads]))
+        nbytes += s.scored_bytes()
+        del lt
+    return layers, nbytes, "q,k,v,o linear layers of one Llama-70B-shaped block (R=2 x 4096 tokens, bf16)"
+
+
+def time_oracle(layers, threads: int, low_fmts):
+    """One pass of the oracle (amax, scales, cast, error, weighting, sums, layer
+    combine) over the sample; independent segments run on host threads."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import ampq_oracle as orc
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        amaxes = list(ex.map(lambda a: orc.amax(a), [v for _, vals, _ in layers for v in vals]))
+        jobs = []
+        for li, (spec, vals, grads) in enumerate(layers):
+            for k, op in enumerate((spec.op0, spec.op1)):
+                a = amaxes[2 * li + k]
+                sc_iv = [orc.scales(f, a) for f in low_fmts]
+                sc = [x[0] for x in sc_iv]
+                iv = [x[1] for x in sc_iv]
+                v = vals[k].reshape(spec.R, -1) if op.per_sample else vals[k].reshape(1, -1)
+                g = grads[k].reshape(spec.R, -1)
+                for r in range(spec.R):
+                    jobs.append((li, k, r, v[r if op.per_sample else 0], g[r], sc, iv))
+        segs = list(ex.map(lambda j: orc.score_segment(j[3], j[4], low_fmts, j[5], j[6]), jobs))
+    import numpy as np
+
+    out = []
+    for li, (spec, _, _) in enumerate(layers):
+        seg = [[None] * spec.R, [None] * spec.R]
+        for j, s in zip(jobs, segs):
+            if j[0] == li:
+                seg[j[1]][j[2]] = s
+        out.append(orc.layer_combine(np.stack(seg[0]), np.stack(seg[1]), [orc.FMT_BASE] + list(low_fmts)))
+    return time.perf_counter() - t0, len(jobs), out
+
+
+def usable_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+
+    low = {"e4m3": [1], "e5m2": [2], "both": [1, 2]}[args.formats]
+    threads = args.cpu_threads or usable_cores()
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    layers, nbytes, desc = oracle_sample(threads, low, dev)
+    for _ in range(max(0, min(args.warmup, 1))):  # a warm-up pass of a deterministic CPU loop buys nothing more
+        time_oracle(layers, threads, low)
+    times = []
+    used = 0
+    for _ in range(args.steps):
+        dt, njobs, _ = time_oracle(layers, threads, low)
+        used = min(threads, njobs)
+        times.append(dt)
+    total = sum(times)
+    val = nbytes * len(times) / total / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama70b_shaped", "sample": desc, "formats": args.formats},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": used, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------
+def run_b200(args):
+    import torch
+
+    from paper_2505_13060_b200 import binding as ampq
+    from paper_2505_13060_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    fmts = {"e4m3": [0, 1], "e5m2": [0, 2], "both": [0, 1, 2]}[args.formats]
+
+    # ---- resident slots: full 70B-shaped blocks of distinct random tensors
+    specs = synth.llama70b_block() if args.workload == "llama70b" else synth.llama7b_block()
+    block_gb = sum(sp.scored_bytes() for sp in specs) / 1e9
+    nres = max(1, min(args.resident_blocks, args.blocks))
+    slots = []
+    for s in range(nres):
+        slots.append([synth.make_layer(sp, dev, seed=100 + rank, layer=7 * s + i) for i, sp in enumerate(specs)])
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream(device=dev)
+    ctx = ampq.Context(local_rank, stream.cuda_stream)
+    ctx.set_formats(fmts)
+    ids = []
+    scored_bytes = 0
+    for b in range(args.blocks):
+        for i, sp in enumerate(specs):
+            lid = ctx.register_layer(sp.kind, "blk%d.%s" % (b, sp.name), sp.R)
+            ampq.bind_layer_tensors(ctx, lid, slots[b % nres][i])
+            ids.append(lid)
+            scored_bytes += sp.scored_bytes()
+    value_bytes = args.blocks * sum(sp.value_bytes() for sp in specs)
+    ctx.set_timing(True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        ctx.score()
+    ctx.get_layer(ids[0])
+    launches_per_step = ctx.last_launch_count()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ev0 = torch.cuda.Event(enable_timing=True)
+    ev1 = torch.cuda.Event(enable_timing=True)
+    score_ms, amax_ms = [], []
+    barrier()
+    if sampler:
+        sampler.start()
+    with torch.cuda.stream(stream):
+        ev0.record(stream)
+        for _ in range(args.steps):
+            ctx.score()
+            t = ctx.get_timing()  # synchronises the step; the per-kernel events are the library's own
+            score_ms.append(t["score_ms"])
+            amax_ms.append(t["amax_ms"])
+        ev1.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * scored_bytes / (ms_per_step * 1e-3) / 1e9
+    first = ctx.get_layer(ids[0])
+
+    # ---- roofline of the dominant kernel (the fused scoring kernel)
+    peak, peak_kind = hbm_peak()
+    k_ms = sum(score_ms) / len(score_ms)
+    achieved = scored_bytes / (k_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "score_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured" else "fallback 6650 GB/s",
+        "traffic": None, "kernel_ms": k_ms, "algorithmic_bytes_per_launch": scored_bytes,
+        "amax_kernel_ms": sum(amax_ms) / len(amax_ms),
+        "amax_kernel_gbs": value_bytes / (sum(amax_ms) / len(amax_ms) * 1e-3) / 1e9,
+        "frac_of_8000_datasheet": achieved / 8000.0,
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "score_kernel_traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            tj = json.load(open(traffic_file))
+            # DRAM bytes per scored byte from an ncu capture of a smaller case, scaled to this launch
+            roofline["traffic"] = tj["dram_bytes_per_scored_byte"][args.formats] * scored_bytes
+            roofline["traffic_source"] = tj["source"]
+        except Exception:
+            pass
+
+    # ---- end to end: tensors in pinned host memory, one block per step
+    e2e = None
+    if not args.no_e2e and rank == 0:
+        ectx = ampq.Context(local_rank, stream.cuda_stream)
+        ectx.set_formats(fmts)
+        host_layers, eids, h2d = [], [], 0
+
+        class H:
+            pass
+
+        for i, sp in enumerate(specs):
+            h = H()
+            h.spec = sp
+            h.values = [t.cpu().pin_memory() for t in slots[0][i].values]
+            h.grads = [t.cpu().pin_memory() for t in slots[0][i].grads]
+            host_layers.append(h)
+            lid = ectx.register_layer(sp.kind, sp.name, sp.R)
+            ampq.bind_layer_tensors(ectx, lid, h, mem=ampq.MEM_HOST)
+            eids.append(lid)
+            h2d += sum(t.numel() * t.element_size() for t in h.values + h.grads)
+        block_scored = sum(sp.scored_bytes() for sp in specs)
+        ectx.score()
+        ectx.get_layer(eids[0])
+        a0 = torch.cuda.Event(enable_timing=True)
+        a1 = torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d2h = 0
+        with torch.cuda.stream(stream):
+            a0.record(stream)
+            for _ in range(args.e2e_steps):
+                ectx.score()
+                res = [ectx.get_layer(l) for l in eids]  # device -> host read of the step's result
+            a1.record(stream)
+        torch.cuda.synchronize()
+        for sp in specs:
+            d2h += 8 * (sp.R + 1 + sp.R * len(fmts) + 2 * len(fmts)) + 2 * (4 + 16 + 4) + 2 * 8 * sp.R * len(fmts)
+        e_ms = a0.elapsed_time(a1) / args.e2e_steps
+        assert res[0]["s_mean"] == ctx.get_layer(ids[0])["s_mean"]
+        e2e = {"value": block_scored / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e_ms,
+               "workload": "one %s-shaped block per step from pinned host memory (AMPQ_MEM_HOST binding)" % args.workload}
+        ectx.destroy()
+        del host_layers
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only
+    cpu = None
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        threads = args.cpu_threads or usable_cores()
+        layers, nbytes, desc = oracle_sample(threads, fmts[1:], dev)
+        dt, njobs, out = time_oracle(layers, threads, fmts[1:])
+        cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": min(threads, njobs), "kind": "oracle",
+               "sample": desc + ", %.2f GB scored in %.1f s" % (nbytes / 1e9, dt)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": args.workload + "_shaped", "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
+                "tokens_per_sample": specs[0].op0.shape[1], "operand_dtype": "bf16", "formats": args.formats,
+                "scored_bytes_per_step_per_gpu": scored_bytes, "resident_blocks": nres,
+                "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block" % (nres, block_gb),
+                "l2": "inputs larger than L2 (%.1f GB resident, 126 MB L2)" % (nres * block_gb),
+                "parallelism": "independent layers per GPU, no data-path collective",
+            },
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu,
+            "check": {"s_mean_layer0": first["s_mean"], "d_meas_layer0": float(first["d_meas"][1])},
+            "pct_of_hbm_peak": {"measured_%.0f" % peak: 100.0 * value / peak, "datasheet_8000": 100.0 * value / 8000.0},
+        }
+        print(json.dumps(line), flush=True)
+    ctx.destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_b200(args)
+
+
+if __name__ == "__main__":
+    main()

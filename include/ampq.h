@@ -127,6 +127,14 @@ int ampq_score(ampq_ctx *ctx);
 /* Number of kernel launches issued by the last ampq_score (diagnostics). */
 int ampq_last_launch_count(const ampq_ctx *ctx);
 
+/* Optional device timing of the kernels of a score.  With timing on, ampq_score
+ * records CUDA events on its stream around the amax kernel, the scoring kernel
+ * and the whole call; ampq_get_timing (synchronises) writes ms[3] = {amax
+ * kernel, scoring kernel, whole score including staging copies and read-back}
+ * of the last score, in milliseconds.  Off by default. */
+int ampq_set_timing(ampq_ctx *ctx, int on);
+int ampq_get_timing(ampq_ctx *ctx, float *ms);
+
 /* Results of one layer after ampq_score (synchronises the stream on the first
  * call after a score).  Any output pointer may be NULL.  Host pointers.
  *   amax[2]                 per operand

@@ -30,7 +30,7 @@ ERR_NONFINITE, ERR_INFEASIBLE, ERR_TOO_LARGE, ERR_NOMEM = -5, -6, -7, -8
 EXPORTS = [
     "ampq_strerror", "ampq_last_error", "ampq_create", "ampq_destroy", "ampq_set_formats",
     "ampq_register_layer", "ampq_bind_operand", "ampq_set_amax", "ampq_score",
-    "ampq_last_launch_count", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
+    "ampq_last_launch_count", "ampq_set_timing", "ampq_get_timing", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
     "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables",
 ]
@@ -68,6 +68,8 @@ def lib():
     L.ampq_set_amax.argtypes = [vp, i, i, C.c_float]
     L.ampq_score.argtypes = [vp]
     L.ampq_last_launch_count.argtypes = [vp]
+    L.ampq_set_timing.argtypes = [vp, i]
+    L.ampq_get_timing.argtypes = [vp, fp]
     L.ampq_get_layer.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, vp, vp]
     L.ampq_get_operand.argtypes = [vp, i, i, vp]
     L.ampq_export_codes.argtypes = [vp, i, i, i, vp]
@@ -170,6 +172,15 @@ class Context:
 
     def last_launch_count(self) -> int:
         return lib().ampq_last_launch_count(self._h)
+
+    def set_timing(self, on: bool):
+        self._check(lib().ampq_set_timing(self._h, 1 if on else 0))
+
+    def get_timing(self) -> dict:
+        """Device milliseconds of the last score: amax kernel, scoring kernel, whole call."""
+        ms = (C.c_float * 3)()
+        self._check(lib().ampq_get_timing(self._h, ms))
+        return dict(amax_ms=ms[0], score_ms=ms[1], total_ms=ms[2])
 
     def get_layer(self, layer_id: int, allow_nonfinite: bool = False) -> dict:
         R, F = self._R[layer_id], self.F

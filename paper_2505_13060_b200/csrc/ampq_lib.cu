@@ -131,6 +131,10 @@ struct ampq_ctx {
     PinBuf<int> h_flags;
     PinBuf<double> h_seg_out, h_layer_out;
     PinBuf<LaunchStatus> h_status;
+
+    bool timing = false;            // record CUDA events around the kernels of a score
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool ev_valid = false;
 };
 
 namespace {
@@ -407,6 +411,8 @@ int ampq_destroy(ampq_ctx* ctx) {
         ctx->d_layer_out.release(); ctx->d_status.release();
         ctx->h_amax_bits.release(); ctx->h_scales.release(); ctx->h_flags.release();
         ctx->h_seg_out.release(); ctx->h_layer_out.release(); ctx->h_status.release();
+        for (int i = 0; i < 6; ++i)
+            if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
     }
     delete ctx;
     return AMPQ_OK;
@@ -498,20 +504,27 @@ int ampq_score(ampq_ctx* ctx) {
     const int nacc = ctx->F;  // S plus one D per low-precision format
     cudaStream_t st = ctx->stream;
     ctx->launches = 0;
+    ctx->ev_valid = false;
+    const bool tm = ctx->timing && T > 0;
+    if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[0], st), "cudaEventRecord");
     if ((rc = stage_host_operands(ctx))) return rc;
     if (T > 0) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
         ++ctx->launches;
+        if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[1], st), "cudaEventRecord");
         if (ctx->namax_tiles > 0) {
             AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
             ++ctx->launches;
         }
+        if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
         AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st), "scales");
         ++ctx->launches;
+        if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         if (ctx->ntiles > 0) {
             AMPQ_CUDA(launch_score(ctx->d_tens.p, ctx->d_tile_begin.p, T, ctx->ntiles, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, st), "score");
             ++ctx->launches;
         }
+        if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");
         AMPQ_CUDA(launch_finalize(ctx->d_segs.p, S, nacc, ctx->d_partials.p, ctx->d_seg_out.p, st), "finalize");
         ++ctx->launches;
         CombineParams prm{};
@@ -528,6 +541,10 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaMemcpyAsync(ctx->h_seg_out.p, ctx->d_seg_out.p, (size_t)S * nacc * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H segments");
         AMPQ_CUDA(cudaMemcpyAsync(ctx->h_layer_out.p, ctx->d_layer_out.p, (size_t)ctx->layer_out_doubles * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H layers");
         AMPQ_CUDA(cudaMemcpyAsync(ctx->h_status.p, ctx->d_status.p, sizeof(LaunchStatus), cudaMemcpyDeviceToHost, st), "D2H status");
+        if (tm) {
+            AMPQ_CUDA(cudaEventRecord(ctx->ev[5], st), "cudaEventRecord");
+            ctx->ev_valid = true;
+        }
     }
     ctx->scored = true;
     ctx->pending = T > 0;
@@ -535,6 +552,30 @@ int ampq_score(ampq_ctx* ctx) {
 }
 
 int ampq_last_launch_count(const ampq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int ampq_set_timing(ampq_ctx* ctx, int on) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    if (on && !ctx->ev[0]) {
+        for (int i = 0; i < 6; ++i) AMPQ_CUDA(cudaEventCreate(&ctx->ev[i]), "cudaEventCreate");
+    }
+    ctx->timing = on != 0;
+    ctx->ev_valid = false;
+    return AMPQ_OK;
+}
+
+int ampq_get_timing(ampq_ctx* ctx, float* ms) {
+    if (!ctx || !ms) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    int rc = sync_results(ctx);
+    if (rc) return rc;
+    if (!ctx->ev_valid) return fail(ctx, AMPQ_ERR_STATE, "timing was not enabled for the last score");
+    AMPQ_CUDA(cudaEventSynchronize(ctx->ev[5]), "cudaEventSynchronize");
+    AMPQ_CUDA(cudaEventElapsedTime(&ms[0], ctx->ev[1], ctx->ev[2]), "cudaEventElapsedTime");
+    AMPQ_CUDA(cudaEventElapsedTime(&ms[1], ctx->ev[3], ctx->ev[4]), "cudaEventElapsedTime");
+    AMPQ_CUDA(cudaEventElapsedTime(&ms[2], ctx->ev[0], ctx->ev[5]), "cudaEventElapsedTime");
+    return AMPQ_OK;
+}
 
 int ampq_get_layer(ampq_ctx* ctx, int layer_id, float* amax, float* scale, float* inv_scale,
                    double* s_per_sample, double* s_mean, double* d_meas_per_sample, double* d_model,
