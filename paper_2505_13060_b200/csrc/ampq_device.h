@@ -5,8 +5,18 @@
 
 namespace ampq {
 
+#ifndef AMPQ_TILE_ELEMS
+#define AMPQ_TILE_ELEMS 524288
+#endif
+#ifndef AMPQ_AMAX_TILE_ELEMS
+#define AMPQ_AMAX_TILE_ELEMS 32768
+#endif
+
 constexpr int kThreads = 256;          // threads per CTA in every streaming kernel
-constexpr int kTileElems = 32768;      // elements of one tile (one CTA's unit of work)
+constexpr int kSubElems = 32768;       // elements between two flushes of the fp32 accumulators into fp64
+constexpr int kTileElems = AMPQ_TILE_ELEMS;           // elements of one scoring tile (one CTA's unit of work)
+constexpr int kAmaxTileElems = AMPQ_AMAX_TILE_ELEMS;  // elements of one amax tile
+static_assert(kTileElems % kSubElems == 0, "a scoring tile is a whole number of flush blocks");
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
 constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
@@ -28,7 +38,7 @@ struct Tensor {
     int R;                   // calibration samples
     int per_sample;          // 1: values are [R, seg_len]; 0: shared by all samples
     int dtype;               // AMPQ_F32 / AMPQ_BF16
-    int rgroups;             // shared values: ceil(R / kMaxRB) tiles per value tile; else 1
+    int rgroups;             // unused by the kernels (kept for table dumps): ceil(R / kMaxRB) or 1
     int seg_base;            // index of segment (this tensor, r = 0) in the segment outputs
     float amax_preset;       // >= 0: use instead of measuring
     int pad;

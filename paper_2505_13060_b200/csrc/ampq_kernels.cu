@@ -1,8 +1,8 @@
 // CUDA kernels of the loss-MSE sensitivity pass for sm_100a.
 //
 // The pass is a stream-reduce: every operand element and its gradient are read
-// once from HBM, all arithmetic happens in registers, and a few floats per
-// 32768-element tile are written back.  The kernels are therefore shaped for
+// once from HBM, all arithmetic happens in registers, and a few doubles per
+// tile (half a million elements) are written back.  The kernels are therefore shaped for
 // HBM bandwidth: 128-bit coalesced non-allocating loads, several independent
 // loads in flight per thread, packed two-wide fp32 arithmetic (fma.rn.f32x2)
 // and the hardware FP8 converts so that the instruction count per element stays
@@ -131,9 +131,9 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
     const long long tile = blockIdx.x;
     const int t = find_tensor(tile_begin, T, tile, &s_slot);
     const Tensor& tn = tens[t];
-    const long long first = (tile - __ldg(tile_begin + t)) * (long long)kTileElems;
+    const long long first = (tile - __ldg(tile_begin + t)) * (long long)kAmaxTileElems;
     const long long left = tn.numel - first;
-    const int n = left < kTileElems ? (int)left : kTileElems;
+    const int n = left < kAmaxTileElems ? (int)left : kAmaxTileElems;
     const int es = tn.dtype == 0 ? 4 : 2;
     const char* base = reinterpret_cast<const char*>(tn.values) + first * es;
     unsigned m = 0;  // fp32 bit pattern of the running max |x|
@@ -323,8 +323,8 @@ __device__ __forceinline__ void score_tile(const char* vbase, const char* const 
 // CTA-wide sum of RB*NACC values in a fixed order; thread a < RB*NACC writes
 // partial (r, a) of the tile.
 template <int NACC, int RB>
-__device__ __forceinline__ void reduce_and_store(Acc<NACC> (&acc)[RB], float* s_red,
-                                                 float* __restrict__ partials, long long slot0,
+__device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], double* s_red,
+                                                 double* __restrict__ partials, long long slot0,
                                                  long long slot_stride) {
     constexpr int NV = RB * NACC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -332,7 +332,7 @@ __device__ __forceinline__ void reduce_and_store(Acc<NACC> (&acc)[RB], float* s_
     for (int r = 0; r < RB; ++r) {
 #pragma unroll
         for (int a = 0; a < NACC; ++a) {
-            float x = acc[r].v[a].x + acc[r].v[a].y;
+            double x = acc[r][a];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
             if (lane == 0) s_red[warp * NV + r * NACC + a] = x;
@@ -340,7 +340,7 @@ __device__ __forceinline__ void reduce_and_store(Acc<NACC> (&acc)[RB], float* s_
     }
     __syncthreads();
     if (threadIdx.x < NV) {
-        float x = 0.0f;
+        double x = 0.0;
 #pragma unroll
         for (int w = 0; w < kThreads / 32; ++w) x += s_red[w * NV + threadIdx.x];
         const int r = threadIdx.x / NACC, a = threadIdx.x % NACC;
@@ -348,33 +348,57 @@ __device__ __forceinline__ void reduce_and_store(Acc<NACC> (&acc)[RB], float* s_
     }
 }
 
+// One scoring tile: blocks of kSubElems elements are summed in fp32 per thread
+// (at most kSubElems / kThreads terms per accumulator lane) and each block's
+// sums are added to per-thread fp64 accumulators, so the length of a tile does
+// not cost accuracy.
 template <int DT, int FMASK, int RB>
 __device__ __forceinline__ void score_tile_and_store(const Tensor& tn, long long voff, long long goff,
                                                      int r0, int n, const float2 (&inv2)[2],
-                                                     const float2 (&nsc2)[2], float* s_red,
-                                                     float* __restrict__ partials, long long slot0) {
+                                                     const float2 (&nsc2)[2], double* s_red,
+                                                     double* __restrict__ partials, long long slot0) {
     constexpr int NACC = Fm<FMASK>::kAcc;
-    Acc<NACC> acc[RB];
+    double acc64[RB][NACC];
 #pragma unroll
     for (int r = 0; r < RB; ++r)
 #pragma unroll
-        for (int a = 0; a < NACC; ++a) acc[r].v[a] = make_float2(0.0f, 0.0f);
+        for (int a = 0; a < NACC; ++a) acc64[r][a] = 0.0;
     const int es = Elem<DT>::kBytes;
     const char* vbase = reinterpret_cast<const char*>(tn.values) + voff * es;
     const char* gbase[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r)
         gbase[r] = reinterpret_cast<const char*>(tn.grads) + (goff + (long long)(r0 + r) * tn.grad_stride) * es;
-    score_tile<DT, FMASK, RB>(vbase, gbase, n, inv2, nsc2, acc);
-    reduce_and_store<NACC, RB>(acc, s_red, partials, slot0, tn.tiles_per_seg);
+    for (int sub = 0; sub < n; sub += kSubElems) {
+        Acc<NACC> acc[RB];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) acc[r].v[a] = make_float2(0.0f, 0.0f);
+        const int m = n - sub < kSubElems ? n - sub : kSubElems;
+        const char* gsub[RB];
+#pragma unroll
+        for (int r = 0; r < RB; ++r) gsub[r] = gbase[r] + (long long)sub * es;
+        score_tile<DT, FMASK, RB>(vbase + (long long)sub * es, gsub, m, inv2, nsc2, acc);
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) acc64[r][a] += (double)acc[r].v[a].x + (double)acc[r].v[a].y;
+    }
+    reduce_and_store<NACC, RB>(acc64, s_red, partials, slot0, tn.tiles_per_seg);
 }
 
-template <int FMASK>
+// One launch per sample-group size RB (1..4): tiles of per-sample operands and
+// the single-sample remainder of shared operands run with RB = 1; shared
+// operands (weights) are read once per group of up to four samples, whose
+// gradients are weighted against the same registers.  Separate launches keep
+// the register budget of the common RB = 1 case small.
+template <int FMASK, int RB>
 __global__ void __launch_bounds__(kThreads)
 score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
-             const float* __restrict__ scales, float* __restrict__ partials) {
+             const float* __restrict__ scales, double* __restrict__ partials) {
     __shared__ int s_slot;
-    __shared__ float s_red[(kThreads / 32) * kMaxRB * kMaxAcc];
+    __shared__ double s_red[(kThreads / 32) * RB * Fm<FMASK>::kAcc];
     const long long tile = blockIdx.x;
     const int t = find_tensor(tile_begin, T, tile, &s_slot);
     const Tensor& tn = tens[t];
@@ -387,55 +411,44 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         inv2[s] = make_float2(iv, iv);
         nsc2[s] = make_float2(-sc, -sc);
     }
-    int i, r0, rb;  // value tile within the segment, first sample, samples in this tile
+    int i, r0;  // value tile within the segment, first sample of this tile
     long long voff;
-    if (tn.per_sample) {
+    if (tn.per_sample) {  // RB == 1
         r0 = local / tn.tiles_per_seg;
         i = local - r0 * tn.tiles_per_seg;
-        rb = 1;
         voff = (long long)r0 * tn.seg_len + (long long)i * kTileElems;
-    } else {
-        i = local / tn.rgroups;
-        r0 = (local - i * tn.rgroups) * kMaxRB;
-        rb = min(kMaxRB, tn.R - r0);
+    } else if (RB == kMaxRB) {  // full groups of four samples
+        const int nfull = tn.R / kMaxRB;
+        i = local / nfull;
+        r0 = (local - i * nfull) * kMaxRB;
+        voff = (long long)i * kTileElems;
+    } else {  // the remainder group: the last R mod 4 samples
+        i = local;
+        r0 = (tn.R / kMaxRB) * kMaxRB;
         voff = (long long)i * kTileElems;
     }
     const long long goff = (long long)i * kTileElems;  // offset inside a sample's gradient
     const long long left = tn.seg_len - (long long)i * kTileElems;
     const int n = left < kTileElems ? (int)left : kTileElems;
     const long long slot0 = tn.partial_base + (long long)r0 * tn.tiles_per_seg + i;
-#define AMPQ_TILE(DT, RB) \
-    score_tile_and_store<DT, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0)
-    if (tn.dtype == 0) {
-        switch (rb) {
-            case 1: AMPQ_TILE(0, 1); break;
-            case 2: AMPQ_TILE(0, 2); break;
-            case 3: AMPQ_TILE(0, 3); break;
-            default: AMPQ_TILE(0, 4); break;
-        }
-    } else {
-        switch (rb) {
-            case 1: AMPQ_TILE(1, 1); break;
-            case 2: AMPQ_TILE(1, 2); break;
-            case 3: AMPQ_TILE(1, 3); break;
-            default: AMPQ_TILE(1, 4); break;
-        }
-    }
-#undef AMPQ_TILE
+    if (tn.dtype == 0)
+        score_tile_and_store<0, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0);
+    else
+        score_tile_and_store<1, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0);
 }
 
 // ---------------------------------------------------------------------------
 // ordered fp64 combine of the per-tile partials: one warp per segment, lane j
 // sums slots j, j+32, ... in order, then a fixed shuffle tree.
 __global__ void finalize_kernel(const Segment* __restrict__ segs, int nseg, int nacc,
-                                const float* __restrict__ partials, double* __restrict__ seg_out) {
+                                const double* __restrict__ partials, double* __restrict__ seg_out) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= nseg) return;
     const Segment sg = segs[warp];
     for (int a = 0; a < nacc; ++a) {
         double x = 0.0;
-        for (int j = lane; j < sg.count; j += 32) x += (double)partials[(sg.first_slot + j) * nacc + a];
+        for (int j = lane; j < sg.count; j += 32) x += partials[(sg.first_slot + j) * nacc + a];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
         if (lane == 0) seg_out[(long long)warp * nacc + a] = x;
@@ -522,20 +535,32 @@ cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* sc
     return cudaGetLastError();
 }
 
-cudaError_t launch_score(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int fmask,
-                         const float* scales, float* partials, cudaStream_t st) {
+template <int RB>
+static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                                   int fmask, const float* scales, double* partials, cudaStream_t st) {
     if (ntiles <= 0) return cudaSuccess;
     const unsigned grid = (unsigned)ntiles;
     switch (fmask) {
-        case 1: score_kernel<1><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
-        case 2: score_kernel<2><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
-        case 3: score_kernel<3><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        case 1: score_kernel<1, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        case 2: score_kernel<2, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
+        case 3: score_kernel<3, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
 }
 
-cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const float* partials, double* seg_out,
+cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                         int fmask, const float* scales, double* partials, cudaStream_t st) {
+    switch (rb) {
+        case 1: return launch_score_rb<1>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
+        case 2: return launch_score_rb<2>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
+        case 3: return launch_score_rb<3>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
+        case 4: return launch_score_rb<4>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const double* partials, double* seg_out,
                             cudaStream_t st) {
     if (nseg <= 0) return cudaSuccess;
     const int warps_per_block = 8;

@@ -20,9 +20,10 @@ cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, 
                         unsigned* amax_bits, cudaStream_t st);
 cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
                           LaunchStatus* status, cudaStream_t st);
-cudaError_t launch_score(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int fmask,
-                         const float* scales, float* partials, cudaStream_t st);
-cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const float* partials, double* seg_out,
+// One launch per sample-group size rb = 1..kMaxRB, each with its own tile table.
+cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                         int fmask, const float* scales, double* partials, cudaStream_t st);
+cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const double* partials, double* seg_out,
                             cudaStream_t st);
 cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParams& prm, const double* seg_out,
                            double* layer_out, cudaStream_t st);

@@ -110,19 +110,20 @@ struct ampq_ctx {
 
     // tables of the last score (host copies)
     std::vector<Tensor> tens;
-    std::vector<long long> tile_begin, amax_tile_begin;
+    std::vector<long long> tile_begin[kMaxRB], amax_tile_begin;  // tile_begin[rb-1]: tiles scored with rb samples
     std::vector<Segment> segs;
     std::vector<Layer> lay;
     std::vector<int> scored_layer_ids;
-    long long ntiles = 0, namax_tiles = 0, nslots = 0;
+    long long ntiles[kMaxRB] = {0, 0, 0, 0}, namax_tiles = 0, nslots = 0;
     int layer_out_doubles = 0;
 
     DevBuf<Tensor> d_tens;
-    DevBuf<long long> d_tile_begin, d_amax_tile_begin;
+    DevBuf<long long> d_tile_begin[kMaxRB], d_amax_tile_begin;
     DevBuf<Segment> d_segs;
     DevBuf<Layer> d_lay;
     DevBuf<unsigned> d_amax_bits;
-    DevBuf<float> d_scales, d_partials;
+    DevBuf<float> d_scales;
+    DevBuf<double> d_partials;
     DevBuf<int> d_flags;
     DevBuf<double> d_seg_out, d_layer_out;
     DevBuf<LaunchStatus> d_status;
@@ -174,10 +175,11 @@ long long extent_of(const LayerRec& l, const Operand& o) { return o.per_sample ?
 
 // Builds the host tables for every layer whose two operands are bound.
 int build_tables(ampq_ctx* ctx) {
-    ctx->tens.clear(); ctx->tile_begin.clear(); ctx->amax_tile_begin.clear();
+    ctx->tens.clear(); ctx->amax_tile_begin.clear();
+    for (auto& tb : ctx->tile_begin) tb.clear();
     ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
     for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
-    long long tiles = 0, atiles = 0, slots = 0;
+    long long tiles[kMaxRB] = {0, 0, 0, 0}, atiles = 0, slots = 0;
     int out_off = 0;
     for (size_t li = 0; li < ctx->layers.size(); ++li) {
         LayerRec& l = ctx->layers[li];
@@ -221,12 +223,22 @@ int build_tables(ampq_ctx* ctx) {
             t.partial_base = slots;
             t.seg_base = (int)ctx->segs.size();
             t.amax_preset = o.amax_preset;
-            const long long my_tiles = o.per_sample ? (long long)l.R * t.tiles_per_seg
-                                                    : (long long)t.tiles_per_seg * t.rgroups;
-            const long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kTileElems - 1) / kTileElems;
-            ctx->tile_begin.push_back(tiles);
+            // per-sample operands: one single-sample tile per (sample, value tile);
+            // shared operands: value tiles x full groups of kMaxRB samples, plus one
+            // remainder group of R mod kMaxRB samples
+            long long my_tiles[kMaxRB] = {0, 0, 0, 0};
+            if (o.per_sample) {
+                my_tiles[0] = (long long)l.R * t.tiles_per_seg;
+            } else {
+                my_tiles[kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
+                if (l.R % kMaxRB) my_tiles[l.R % kMaxRB - 1] += t.tiles_per_seg;
+            }
+            const long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
+            for (int c = 0; c < kMaxRB; ++c) {
+                ctx->tile_begin[c].push_back(tiles[c]);
+                tiles[c] += my_tiles[c];
+            }
             ctx->amax_tile_begin.push_back(atiles);
-            tiles += my_tiles;
             atiles += my_atiles;
             for (int r = 0; r < l.R; ++r) {
                 Segment s{};
@@ -244,13 +256,17 @@ int build_tables(ampq_ctx* ctx) {
         ctx->lay.push_back(ly);
         ctx->scored_layer_ids.push_back((int)li);
     }
-    ctx->tile_begin.push_back(tiles);
+    long long most = atiles;
+    for (int c = 0; c < kMaxRB; ++c) {
+        ctx->tile_begin[c].push_back(tiles[c]);
+        ctx->ntiles[c] = tiles[c];
+        if (tiles[c] > most) most = tiles[c];
+    }
     ctx->amax_tile_begin.push_back(atiles);
-    ctx->ntiles = tiles;
     ctx->namax_tiles = atiles;
     ctx->nslots = slots;
     ctx->layer_out_doubles = out_off;
-    if (tiles > 0x7FFFFFFFLL || atiles > 0x7FFFFFFFLL)
+    if (most > 0x7FFFFFFFLL)
         return fail(ctx, AMPQ_ERR_TOO_LARGE, "more than 2^31-1 tiles in one score");
     return AMPQ_OK;
 }
@@ -259,7 +275,7 @@ int upload_tables(ampq_ctx* ctx) {
     const size_t T = ctx->tens.size(), L = ctx->lay.size(), S = ctx->segs.size();
     const int nacc = 1 + (ctx->F - 1);
     AMPQ_CUDA(ctx->d_tens.ensure(T), "cudaMalloc(tensors)");
-    AMPQ_CUDA(ctx->d_tile_begin.ensure(T + 1), "cudaMalloc(tile_begin)");
+    for (int c = 0; c < kMaxRB; ++c) AMPQ_CUDA(ctx->d_tile_begin[c].ensure(T + 1), "cudaMalloc(tile_begin)");
     AMPQ_CUDA(ctx->d_amax_tile_begin.ensure(T + 1), "cudaMalloc(amax_tile_begin)");
     AMPQ_CUDA(ctx->d_segs.ensure(S), "cudaMalloc(segments)");
     AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
@@ -281,7 +297,8 @@ int upload_tables(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tens.p, ctx->tens.data(), T * sizeof(Tensor), cudaMemcpyHostToDevice, st), "H2D tensors");
         AMPQ_CUDA(cudaMemsetAsync(ctx->d_scales.p, 0, T * 2 * kMaxLow * sizeof(float), st), "memset scales");
     }
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tile_begin.p, ctx->tile_begin.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D tile_begin");
+    for (int c = 0; c < kMaxRB; ++c)
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tile_begin[c].p, ctx->tile_begin[c].data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D tile_begin");
     AMPQ_CUDA(cudaMemcpyAsync(ctx->d_amax_tile_begin.p, ctx->amax_tile_begin.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D amax_tile_begin");
     if (S) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_segs.p, ctx->segs.data(), S * sizeof(Segment), cudaMemcpyHostToDevice, st), "H2D segments");
     if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
@@ -405,7 +422,8 @@ int ampq_destroy(ampq_ctx* ctx) {
         for (auto& l : ctx->layers)
             for (int k = 0; k < 2; ++k)
                 if (l.op[k].stage) cudaFree(l.op[k].stage);
-        ctx->d_tens.release(); ctx->d_tile_begin.release(); ctx->d_amax_tile_begin.release();
+        ctx->d_tens.release(); ctx->d_amax_tile_begin.release();
+        for (auto& b : ctx->d_tile_begin) b.release();
         ctx->d_segs.release(); ctx->d_lay.release(); ctx->d_amax_bits.release(); ctx->d_scales.release();
         ctx->d_partials.release(); ctx->d_flags.release(); ctx->d_seg_out.release();
         ctx->d_layer_out.release(); ctx->d_status.release();
@@ -520,8 +538,9 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st), "scales");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
-        if (ctx->ntiles > 0) {
-            AMPQ_CUDA(launch_score(ctx->d_tens.p, ctx->d_tile_begin.p, T, ctx->ntiles, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, st), "score");
+        for (int c = 0; c < kMaxRB; ++c) {
+            if (ctx->ntiles[c] <= 0) continue;
+            AMPQ_CUDA(launch_score(c + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, st), "score");
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");
