@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--formats", default="e4m3", choices=["e4m3", "e5m2", "both"])
     ap.add_argument("--workload", default="llama70b", choices=["llama70b", "llama7b"],
                     help="llama70b is the benchmark; llama7b (3.2 GB per block) is the small case for profiler captures")
+    ap.add_argument("--layers", default="",
+                    help="comma-separated subset of a block's layers (q,k,v,o,gate,up,down); a small case of the "
+                         "same kernels for profiler captures, never the benchmark")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -237,11 +240,16 @@ def run_b200(args):
 
     # ---- resident slots: full 70B-shaped blocks of distinct random tensors
     specs = synth.llama70b_block() if args.workload == "llama70b" else synth.llama7b_block()
+    if args.layers:
+        keep = args.layers.split(",")
+        specs = [sp for sp in specs if sp.name in keep]
+        if not specs:
+            raise SystemExit("--layers matched no layer of the block")
     block_gb = sum(sp.scored_bytes() for sp in specs) / 1e9
     nres = max(1, min(args.resident_blocks, args.blocks))
     slots = []
     for s in range(nres):
-        slots.append([synth.make_layer(sp, dev, seed=100 + rank, layer=7 * s + i) for i, sp in enumerate(specs)])
+        slots.append([synth.make_layer(sp, dev, seed=100 + rank, layer=len(specs) * s + i) for i, sp in enumerate(specs)])
     torch.cuda.synchronize()
     stream = torch.cuda.Stream(device=dev)
     ctx = ampq.Context(local_rank, stream.cuda_stream)
@@ -373,7 +381,7 @@ def run_b200(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": args.workload + "_shaped", "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
+                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
                 "tokens_per_sample": specs[0].op0.shape[1], "operand_dtype": "bf16", "formats": args.formats,
                 "scored_bytes_per_step_per_gpu": scored_bytes, "resident_blocks": nres,
                 "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block" % (nres, block_gb),
