@@ -195,6 +195,37 @@ int ampq_select_tables(int J, const int *P, const long long *off, const double *
                        const double *d, double budget, int *p_out, double *c_total,
                        double *d_total);
 
+/* The paper has no counterpart of this call; it exists for callers that are
+ * not allowed to allocate device memory: code that runs while another library
+ * owns the device heap through its own pool, code in a phase where a device
+ * allocation would stall or fragment the heap, plug-ins that are handed fixed
+ * buffers.  It runs the same pass as ampq_score (amax, scales, FP8 cast,
+ * error, gradient weighting, per-tile sums, ordered fp64 combine) on ONE
+ * segment -- numel elements of `values` weighted by `grads`, one low-precision
+ * format `fmt` (AMPQ_FMT_E4M3 or AMPQ_FMT_E5M2) -- and calls no cudaMalloc,
+ * cudaFree or other allocating routine: its tables and per-tile partial sums
+ * live in a fixed array in the library's device image (about 64 KiB, held by
+ * every GPU that loads the library until the process exits).
+ *   device, cuda_stream   the device, and a cudaStream_t on it (0 = default)
+ *   values, grads         device pointers, numel elements of `dtype` each,
+ *                         aligned to the element size; borrowed until the work
+ *                         on the stream has finished
+ *   numel                 0 .. AMPQ_NOALLOC_MAX_NUMEL; larger sizes are refused
+ *                         with AMPQ_ERR_TOO_LARGE before anything is launched
+ *   amax                  >= 0: use this amax (static scale); < 0: measure it
+ *   dev_out               device pointer, 3 doubles, 8-byte aligned:
+ *                         {S = sum (z g)^2, D = sum (g (Q(z) - z))^2, amax};
+ *                         S and D are NaN when the operand holds Inf or NaN
+ * Asynchronous on the stream; nothing is copied to the host.  The first call on
+ * a device looks up the array's device address (once per device); make that
+ * first call before any stream capture begins.  Every call on a device uses
+ * the same array and overwrites what the previous call left there, so calls
+ * whose work may overlap on the GPU (different streams, different threads)
+ * race: order them on one stream or with events. */
+#define AMPQ_NOALLOC_MAX_NUMEL 2147483648LL
+int ampq_score_segment_noalloc(int device, void *cuda_stream, int dtype, int fmt, const void *values,
+                               const void *grads, long long numel, float amax, double *dev_out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,8 +32,9 @@ EXPORTS = [
     "ampq_register_layer", "ampq_bind_operand", "ampq_set_amax", "ampq_score",
     "ampq_last_launch_count", "ampq_set_timing", "ampq_get_timing", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
     "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
-    "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables",
+    "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
 ]
+NOALLOC_MAX_NUMEL = 2147483648
 
 _lib = None
 
@@ -80,6 +81,7 @@ def lib():
     L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
     L.ampq_select.argtypes = [vp, i, C.c_double, vp, dp, dp]
     L.ampq_select_tables.argtypes = [i, vp, vp, vp, vp, C.c_double, vp, dp, dp]
+    L.ampq_score_segment_noalloc.argtypes = [i, vp, i, i, vp, vp, ll, C.c_float, vp]
     for name in EXPORTS:
         if name not in ("ampq_strerror", "ampq_last_error"):
             getattr(L, name).restype = i
@@ -118,6 +120,21 @@ def select_tables(c_tables, d_tables, budget: float):
     if rc:
         raise AmpqError(rc)
     return p[:J].copy(), co.value, do.value
+
+
+def score_segment_noalloc(device: int, stream: int, dtype: int, fmt: int, values_ptr: int, grads_ptr: int,
+                          numel: int, amax: float, dev_out_ptr: int):
+    """``ampq_score_segment_noalloc``: the pass over one segment for callers that
+    must not allocate device memory (the library's own fixed device array holds
+    the tables and partial sums).  ``dev_out_ptr`` receives {S, D, amax} as three
+    doubles on the device; asynchronous on ``stream``."""
+    rc = lib().ampq_score_segment_noalloc(device, C.c_void_p(stream), dtype, fmt, C.c_void_p(values_ptr),
+                                          C.c_void_p(grads_ptr), numel, amax, C.c_void_p(dev_out_ptr))
+    if rc == ERR_TOO_LARGE:
+        raise AmpqError(rc, "numel %d exceeds the fixed scratch of the no-allocation call (at most %d elements)"
+                        % (numel, NOALLOC_MAX_NUMEL))
+    if rc:
+        raise AmpqError(rc, "ampq_score_segment_noalloc")
 
 
 class Context:
