@@ -60,7 +60,8 @@ enum {
     AMPQ_ERR_NONFINITE = -5,   /* a scored operand holds Inf or NaN                 */
     AMPQ_ERR_INFEASIBLE = -6,  /* no assignment meets the budget                    */
     AMPQ_ERR_TOO_LARGE = -7,   /* selection exceeded its state limit                */
-    AMPQ_ERR_NOMEM = -8
+    AMPQ_ERR_NOMEM = -8,
+    AMPQ_ERR_TIMEOUT = -9      /* a bounded wait inside a kernel ran out; results invalid */
 };
 
 const char *ampq_strerror(int status);
@@ -119,9 +120,10 @@ int ampq_set_amax(ampq_ctx *ctx, int layer_id, int operand, float amax);
  *   per (tensor, sample): S = sum_k (z_k g_k)^2, D_f = sum_k (g_k e_k)^2;
  *   per layer: s^r = S(op0,r) + S(op1,r), s = mean_r s^r, d_model_f = alpha_f s,
  *   d_meas_f = mean_r (D_f(op0,r) + D_f(op1,r)).
- * Sums are accumulated in fp32 over runs of at most a few hundred terms per
- * thread and combined in a fixed order in fp64, so results are reproducible
- * run to run. */
+ * Sums are accumulated in fp32 over runs of at most 64 terms per lane and
+ * combined in a fixed order in fp64, so results are reproducible run to run.
+ * The scoring kernel's internal waits are bounded: if one ever runs out, the
+ * getters return AMPQ_ERR_TIMEOUT for that score and the context stays usable. */
 int ampq_score(ampq_ctx *ctx);
 
 /* Number of kernel launches issued by the last ampq_score (diagnostics). */

@@ -24,7 +24,7 @@ MEM_DEVICE, MEM_HOST = 0, 1
 
 OK = 0
 ERR_INVALID, ERR_ALIGN, ERR_STATE, ERR_CUDA = -1, -2, -3, -4
-ERR_NONFINITE, ERR_INFEASIBLE, ERR_TOO_LARGE, ERR_NOMEM = -5, -6, -7, -8
+ERR_NONFINITE, ERR_INFEASIBLE, ERR_TOO_LARGE, ERR_NOMEM, ERR_TIMEOUT = -5, -6, -7, -8, -9
 
 # every symbol include/ampq.h declares
 EXPORTS = [

@@ -5,18 +5,24 @@
 
 namespace ampq {
 
-#ifndef AMPQ_TILE_ELEMS
-#define AMPQ_TILE_ELEMS 524288
-#endif
 #ifndef AMPQ_AMAX_TILE_ELEMS
 #define AMPQ_AMAX_TILE_ELEMS 32768
 #endif
 
-constexpr int kThreads = 256;          // threads per CTA in every streaming kernel
-constexpr int kSubElems = 32768;       // elements between two flushes of the fp32 accumulators into fp64
-constexpr int kTileElems = AMPQ_TILE_ELEMS;           // elements of one scoring tile (one CTA's unit of work)
+constexpr int kThreads = 256;          // threads per CTA of the amax kernel
+constexpr int kConsumers = 256;        // scoring threads of a scoring CTA (warps 0..7)
+constexpr int kScoreThreads = kConsumers + 32;  // plus the producer warp that feeds the shared-memory ring
+constexpr int kSubElems = 32768;       // direct path: elements between two flushes of the fp32 accumulators into fp64
+constexpr int kFlushChunks = 8;        // ring path: chunks between two flushes (at most 64 terms per fp32 lane)
+constexpr unsigned kSpinLimit = 1u << 22;  // polls of an mbarrier before a wait gives up
+// A scoring tile (one partial sum per sample and accumulator) holds 2^shift
+// elements of a segment; the host picks the shift per score so that small
+// problems still spread over every SM and large ones pay few tile ends.
+constexpr int kMinTileShift = 15;
+constexpr int kMaxTileShift = 19;
+constexpr int kTileElems = 1 << kMaxTileShift;        // largest scoring tile
 constexpr int kAmaxTileElems = AMPQ_AMAX_TILE_ELEMS;  // elements of one amax tile
-static_assert(kTileElems % kSubElems == 0, "a scoring tile is a whole number of flush blocks");
+static_assert((1 << kMinTileShift) % kSubElems == 0, "a scoring tile is a whole number of flush blocks");
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
 constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
@@ -34,7 +40,7 @@ struct Tensor {
     long long seg_len;       // elements of one segment: numel/R (per-sample) or numel (shared)
     long long grad_stride;   // elements between consecutive samples' gradients
     long long partial_base;  // partial slot of (r, i) = partial_base + r*tiles_per_seg + i
-    int tiles_per_seg;       // ceil(seg_len / kTileElems)
+    int tiles_per_seg;       // ceil(seg_len / tile elements of this score)
     int R;                   // calibration samples
     int per_sample;          // 1: values are [R, seg_len]; 0: shared by all samples
     int dtype;               // AMPQ_F32 / AMPQ_BF16
@@ -64,6 +70,7 @@ inline int layer_block_doubles(int R, int F) { return R + 1 + R * F + 2 * F; }
 
 struct LaunchStatus {
     int nonfinite;  // set when some tensor's amax is Inf/NaN
+    int timeout;    // set when a wait inside the scoring kernel ran out
 };
 
 }  // namespace ampq

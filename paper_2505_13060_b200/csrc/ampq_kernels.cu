@@ -2,9 +2,11 @@
 //
 // The pass is a stream-reduce: every operand element and its gradient are read
 // once from HBM, all arithmetic happens in registers, and a few doubles per
-// tile (half a million elements) are written back.  The kernels are therefore shaped for
-// HBM bandwidth: 128-bit coalesced non-allocating loads, several independent
-// loads in flight per thread, packed two-wide fp32 arithmetic (fma.rn.f32x2)
+// tile are written back.  The kernels are therefore shaped for HBM bandwidth:
+// the scoring kernel is persistent and stages operand and gradient chunks in a
+// shared-memory ring with bulk asynchronous copies (TMA) so that the bytes in
+// flight do not depend on the arithmetic; the amax kernel uses 128-bit
+// coalesced non-allocating loads; packed two-wide fp32 arithmetic (fma.rn.f32x2)
 // and the hardware FP8 converts so that the instruction count per element stays
 // below what 148 SMs can issue at full memory speed.  No tensor cores: there is
 // no contraction anywhere on this path.
@@ -116,7 +118,10 @@ __device__ __forceinline__ int find_tensor(const long long* __restrict__ begin, 
 __global__ void init_amax_kernel(const Tensor* __restrict__ tens, int T,
                                  unsigned* __restrict__ amax_bits, LaunchStatus* status) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t == 0) status->nonfinite = 0;
+    if (t == 0) {
+        status->nonfinite = 0;
+        status->timeout = 0;
+    }
     if (t < T) {
         float p = tens[t].amax_preset;
         amax_bits[t] = (p >= 0.0f) ? __float_as_uint(p) : 0u;
@@ -320,8 +325,70 @@ __device__ __forceinline__ void score_tile(const char* vbase, const char* const 
     }
 }
 
-// CTA-wide sum of RB*NACC values in a fixed order; thread a < RB*NACC writes
-// partial (r, a) of the tile.
+// ---------------------------------------------------------------------------
+// shared-memory ring fed by bulk asynchronous copies (TMA, untiled form)
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) {
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned long long* b, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* b, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* b, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Global -> this CTA's shared memory, completion counted in bytes on an
+// mbarrier.  Both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, unsigned long long* b) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(b))
+                 : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(const void* p) {
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "r"(smem_u32(p)));
+    return r;
+}
+__device__ __forceinline__ void consumer_barrier() {  // the kConsumers scoring threads only
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+
+// Waits for a phase of an mbarrier, at most kSpinLimit polls.  A wait that runs
+// out raises the CTA's abort flag; once that is up every wait returns false at
+// once, so that all threads still walk the same control flow to the end.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* b, unsigned parity, volatile int* s_abort) {
+    if (*s_abort) return false;
+    for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+        if (mbar_try_wait(b, parity)) return true;
+        if ((spin & 255u) == 255u && *s_abort) return false;
+    }
+    *s_abort = 1;
+    return false;
+}
+
+// CTA-wide sum of RB*NACC values in a fixed order over the scoring warps;
+// thread a < RB*NACC writes partial (r, a) of the tile.  s_red holds one
+// kConsumers/32 x RB*NACC block; the caller alternates two blocks from tile to
+// tile so that a tile's readers never meet the next tile's writers.
 template <int NACC, int RB>
 __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], double* s_red,
                                                  double* __restrict__ partials, long long slot0,
@@ -338,37 +405,36 @@ __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], 
             if (lane == 0) s_red[warp * NV + r * NACC + a] = x;
         }
     }
-    __syncthreads();
+    consumer_barrier();
     if (threadIdx.x < NV) {
         double x = 0.0;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) x += s_red[w * NV + threadIdx.x];
+        for (int w = 0; w < kConsumers / 32; ++w) x += s_red[w * NV + threadIdx.x];
         const int r = threadIdx.x / NACC, a = threadIdx.x % NACC;
         partials[(slot0 + r * slot_stride) * NACC + a] = x;
     }
 }
 
-// One scoring tile: blocks of kSubElems elements are summed in fp32 per thread
-// (at most kSubElems / kThreads terms per accumulator lane) and each block's
-// sums are added to per-thread fp64 accumulators, so the length of a tile does
-// not cost accuracy.
+template <int NACC, int RB>
+__device__ __forceinline__ void flush_acc(Acc<NACC> (&acc)[RB], double (&acc64)[RB][NACC]) {
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
+#pragma unroll
+        for (int a = 0; a < NACC; ++a) {
+            acc64[r][a] += (double)acc[r].v[a].x + (double)acc[r].v[a].y;
+            acc[r].v[a] = make_float2(0.0f, 0.0f);
+        }
+}
+
+// n elements straight from global memory (what the ring does not carry: ragged
+// ends and tensors that are not 16-byte aligned), in blocks of kSubElems so that
+// an fp32 accumulator lane never sees more than kSubElems / kConsumers terms.
 template <int DT, int FMASK, int RB>
-__device__ __forceinline__ void score_tile_and_store(const Tensor& tn, long long voff, long long goff,
-                                                     int r0, int n, const float2 (&inv2)[2],
-                                                     const float2 (&nsc2)[2], double* s_red,
-                                                     double* __restrict__ partials, long long slot0) {
+__device__ __forceinline__ void score_direct(const char* vbase, const char* const (&gbase)[RB], int n,
+                                             const float2 (&inv2)[2], const float2 (&nsc2)[2],
+                                             double (&acc64)[RB][Fm<FMASK>::kAcc]) {
     constexpr int NACC = Fm<FMASK>::kAcc;
-    double acc64[RB][NACC];
-#pragma unroll
-    for (int r = 0; r < RB; ++r)
-#pragma unroll
-        for (int a = 0; a < NACC; ++a) acc64[r][a] = 0.0;
     const int es = Elem<DT>::kBytes;
-    const char* vbase = reinterpret_cast<const char*>(tn.values) + voff * es;
-    const char* gbase[RB];
-#pragma unroll
-    for (int r = 0; r < RB; ++r)
-        gbase[r] = reinterpret_cast<const char*>(tn.grads) + (goff + (long long)(r0 + r) * tn.grad_stride) * es;
     for (int sub = 0; sub < n; sub += kSubElems) {
         Acc<NACC> acc[RB];
 #pragma unroll
@@ -380,61 +446,230 @@ __device__ __forceinline__ void score_tile_and_store(const Tensor& tn, long long
 #pragma unroll
         for (int r = 0; r < RB; ++r) gsub[r] = gbase[r] + (long long)sub * es;
         score_tile<DT, FMASK, RB>(vbase + (long long)sub * es, gsub, m, inv2, nsc2, acc);
-#pragma unroll
-        for (int r = 0; r < RB; ++r)
-#pragma unroll
-            for (int a = 0; a < NACC; ++a) acc64[r][a] += (double)acc[r].v[a].x + (double)acc[r].v[a].y;
+        flush_acc<NACC, RB>(acc, acc64);
     }
-    reduce_and_store<NACC, RB>(acc64, s_red, partials, slot0, tn.tiles_per_seg);
 }
 
-// One launch per sample-group size RB (1..4): tiles of per-sample operands and
-// the single-sample remainder of shared operands run with RB = 1; shared
-// operands (weights) are read once per group of up to four samples, whose
-// gradients are weighted against the same registers.  Separate launches keep
-// the register budget of the common RB = 1 case small.
-template <int FMASK, int RB>
-__global__ void __launch_bounds__(kThreads)
-score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
-             const float* __restrict__ scales, double* __restrict__ partials) {
-    __shared__ int s_slot;
-    __shared__ double s_red[(kThreads / 32) * RB * Fm<FMASK>::kAcc];
-    const long long tile = blockIdx.x;
-    const int t = find_tensor(tile_begin, T, tile, &s_slot);
-    const Tensor& tn = tens[t];
-    const int local = (int)(tile - __ldg(tile_begin + t));
-    float2 inv2[2], nsc2[2];
-#pragma unroll
-    for (int s = 0; s < 2; ++s) {
-        float sc = __ldg(scales + t * 2 * kMaxLow + s * 2 + 0);
-        float iv = __ldg(scales + t * 2 * kMaxLow + s * 2 + 1);
-        inv2[s] = make_float2(iv, iv);
-        nsc2[s] = make_float2(-sc, -sc);
-    }
-    int i, r0;  // value tile within the segment, first sample of this tile
-    long long voff;
+// Geometry of the ring for RB gradient streams per value stream.
+template <int RB>
+struct Ring {
+    static constexpr int kU = RB <= 2 ? 2 : 1;                       // 16-byte vectors per thread, stream and chunk
+    static constexpr int kChunkBytes = kU * kConsumers * 16;          // bytes of one stream in one stage
+    static constexpr int kStageBytes = (1 + RB) * kChunkBytes;
+    static constexpr int kStages = RB == 1 ? 6 : (RB == 2 ? 4 : (RB == 3 ? 6 : 4));
+    static constexpr int kRingBytes = kStages * kStageBytes;
+    static constexpr int kRedDoubles = 2 * (kConsumers / 32) * RB * kMaxAcc;
+    // ring | full[kStages] empty[kStages] | reduction blocks | abort flag
+    static constexpr int kSmemBytes = kRingBytes + 2 * kStages * 8 + kRedDoubles * 8 + 16;
+};
+
+// Where a tile lives.
+struct TileGeom {
+    long long voff, goff, slot0;
+    int r0, n;
+};
+
+template <int RB>
+__device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, int tile_shift) {
+    TileGeom q;
+    int i;  // value tile within the segment
     if (tn.per_sample) {  // RB == 1
-        r0 = local / tn.tiles_per_seg;
-        i = local - r0 * tn.tiles_per_seg;
-        voff = (long long)r0 * tn.seg_len + (long long)i * kTileElems;
+        q.r0 = local / tn.tiles_per_seg;
+        i = local - q.r0 * tn.tiles_per_seg;
+        q.voff = (long long)q.r0 * tn.seg_len + ((long long)i << tile_shift);
     } else if (RB == kMaxRB) {  // full groups of four samples
         const int nfull = tn.R / kMaxRB;
         i = local / nfull;
-        r0 = (local - i * nfull) * kMaxRB;
-        voff = (long long)i * kTileElems;
+        q.r0 = (local - i * nfull) * kMaxRB;
+        q.voff = (long long)i << tile_shift;
     } else {  // the remainder group: the last R mod 4 samples
         i = local;
-        r0 = (tn.R / kMaxRB) * kMaxRB;
-        voff = (long long)i * kTileElems;
+        q.r0 = (tn.R / kMaxRB) * kMaxRB;
+        q.voff = (long long)i << tile_shift;
     }
-    const long long goff = (long long)i * kTileElems;  // offset inside a sample's gradient
-    const long long left = tn.seg_len - (long long)i * kTileElems;
-    const int n = left < kTileElems ? (int)left : kTileElems;
-    const long long slot0 = tn.partial_base + (long long)r0 * tn.tiles_per_seg + i;
-    if (tn.dtype == 0)
-        score_tile_and_store<0, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0);
-    else
-        score_tile_and_store<1, FMASK, RB>(tn, voff, goff, r0, n, inv2, nsc2, s_red, partials, slot0);
+    q.goff = (long long)i << tile_shift;  // offset inside a sample's gradient
+    const long long left = tn.seg_len - q.goff;
+    q.n = left < (1LL << tile_shift) ? (int)left : (1 << tile_shift);
+    q.slot0 = tn.partial_base + (long long)q.r0 * tn.tiles_per_seg + i;
+    return q;
+}
+
+// The scoring kernel.  Persistent: CTA b takes tiles b, b + gridDim.x, ... of
+// the launch's tile table.  Warps 0..7 score; warp 8 is the producer: one lane
+// streams every full 16-byte-aligned chunk of the value tile and of its RB
+// gradient tiles into a ring of shared-memory stages with bulk asynchronous
+// copies, running as far ahead as the ring is deep, tile after tile, so that
+// the bytes in flight do not depend on how long the arithmetic of a chunk
+// takes.  A scoring thread takes its 16-byte vectors of a stage into
+// registers, hands the stage back and then does the arithmetic.  fp32 sums are
+// flushed into fp64 every kFlushChunks chunks; a tile ends with the CTA-wide
+// ordered sum and one partial per (sample, accumulator).
+//
+// One launch per sample-group size RB (1..4): per-sample operands and the
+// single-sample remainder of shared operands run with RB = 1; shared operands
+// (weights) are read once per group of up to four samples.
+template <int FMASK, int RB>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
+             int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
+             LaunchStatus* __restrict__ status) {
+    using RG = Ring<RB>;
+    constexpr int NACC = Fm<FMASK>::kAcc;
+    constexpr int U = RG::kU;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* ring = smem;
+    unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + RG::kRingBytes);
+    unsigned long long* empty = full + RG::kStages;
+    double* s_red = reinterpret_cast<double*>(empty + RG::kStages);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_red + RG::kRedDoubles);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < RG::kStages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, kConsumers / 32);
+        }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const bool producer = threadIdx.x >= kConsumers;
+    unsigned it = 0;  // chunks through the ring so far (same count on both sides)
+    int t = 0;        // tensor of the current tile; tiles only move forward
+    if (producer) {
+        if (threadIdx.x == kConsumers) {
+            for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+                while (tile >= __ldg(tile_begin + t + 1)) ++t;
+                const Tensor& tn = tens[t];
+                const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
+                const int es = tn.dtype == 0 ? 4 : 2;
+                const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
+                const char* gb[RB];
+                bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
+                    aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
+                }
+                const int nchunks = aligned ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
+                for (int c = 0; c < nchunks; ++c, ++it) {
+                    const unsigned s = it % RG::kStages, lap = it / RG::kStages;
+                    if (lap > 0 && !mbar_wait(empty + s, (lap - 1) & 1, s_abort)) break;
+                    unsigned char* dst = ring + s * RG::kStageBytes;
+                    mbar_arrive_expect_tx(full + s, RG::kStageBytes);
+                    bulk_load(dst, vb + (long long)c * RG::kChunkBytes, RG::kChunkBytes, full + s);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+                        bulk_load(dst + (1 + r) * RG::kChunkBytes, gb[r] + (long long)c * RG::kChunkBytes,
+                                  RG::kChunkBytes, full + s);
+                }
+                if (*s_abort) break;
+            }
+            if (*s_abort) {
+                // The scoring warps stopped taking stages.  Every copy issued so far
+                // must have landed before the CTA gives its shared memory back:
+                // wait (bounded) for the last lap of each stage.
+                for (unsigned k = 0; k < (unsigned)RG::kStages && k < it; ++k) {
+                    const unsigned j = it - 1 - k;
+                    for (unsigned spin = 0; spin < kSpinLimit; ++spin)
+                        if (mbar_try_wait(full + j % RG::kStages, (j / RG::kStages) & 1)) break;
+                }
+                atomicExch(&status->timeout, 1);
+            }
+        }
+        return;
+    }
+
+    // ---- scoring warps
+    const int tid = threadIdx.x;
+    int red_block = 0;
+    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        while (tile >= __ldg(tile_begin + t + 1)) ++t;
+        const Tensor& tn = tens[t];
+        const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
+        const int es = tn.dtype == 0 ? 4 : 2;
+        float2 inv2[2], nsc2[2];
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const float sc = __ldg(scales + t * 2 * kMaxLow + s * 2 + 0);
+            const float iv = __ldg(scales + t * 2 * kMaxLow + s * 2 + 1);
+            inv2[s] = make_float2(iv, iv);
+            nsc2[s] = make_float2(-sc, -sc);
+        }
+        const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
+        const char* gb[RB];
+        bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
+            aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
+        }
+        const int nchunks = aligned ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
+
+        double acc64[RB][NACC];
+        Acc<NACC> acc[RB];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) {
+                acc64[r][a] = 0.0;
+                acc[r].v[a] = make_float2(0.0f, 0.0f);
+            }
+        for (int c = 0; c < nchunks; ++c, ++it) {
+            const unsigned s = it % RG::kStages, lap = it / RG::kStages;
+            const bool ok = mbar_wait(full + s, lap & 1, s_abort);
+            uint4 v[U], g[RB][U];
+            if (ok) {
+                const unsigned char* st = ring + s * RG::kStageBytes;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    v[u] = lds_v4(st + (u * kConsumers + tid) * 16);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+                        g[r][u] = lds_v4(st + (1 + r) * RG::kChunkBytes + (u * kConsumers + tid) * 16);
+                }
+            }
+            __syncwarp();
+            if (ok && (tid & 31) == 0) mbar_arrive(empty + s);  // the warp's vectors are in registers
+            if (ok) {
+                if (tn.dtype == 0) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        float2 z[2], gg[RB][2];
+                        Elem<0>::unpack(v[u], z);
+#pragma unroll
+                        for (int r = 0; r < RB; ++r) Elem<0>::unpack(g[r][u], gg[r]);
+                        accumulate_pairs<FMASK, RB, 2>(z, gg, inv2, nsc2, acc);
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        float2 z[4], gg[RB][4];
+                        Elem<1>::unpack(v[u], z);
+#pragma unroll
+                        for (int r = 0; r < RB; ++r) Elem<1>::unpack(g[r][u], gg[r]);
+                        accumulate_pairs<FMASK, RB, 4>(z, gg, inv2, nsc2, acc);
+                    }
+                }
+            }
+            if ((c % kFlushChunks) == kFlushChunks - 1) flush_acc<NACC, RB>(acc, acc64);
+        }
+        flush_acc<NACC, RB>(acc, acc64);
+        // what the ring did not carry
+        const int done = (int)(((long long)nchunks * RG::kChunkBytes) / es);
+        if (done < q.n) {
+            const char* gt[RB];
+#pragma unroll
+            for (int r = 0; r < RB; ++r) gt[r] = gb[r] + (long long)done * es;
+            if (tn.dtype == 0)
+                score_direct<0, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
+            else
+                score_direct<1, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
+        }
+        reduce_and_store<NACC, RB>(acc64, s_red + red_block * (kConsumers / 32) * RB * NACC, partials, q.slot0,
+                                   tn.tiles_per_seg);
+        red_block ^= 1;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -535,27 +770,47 @@ cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* sc
     return cudaGetLastError();
 }
 
-template <int RB>
-static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
-                                   int fmask, const float* scales, double* partials, cudaStream_t st) {
-    if (ntiles <= 0) return cudaSuccess;
-    const unsigned grid = (unsigned)ntiles;
-    switch (fmask) {
-        case 1: score_kernel<1, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
-        case 2: score_kernel<2, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
-        case 3: score_kernel<3, RB><<<grid, kThreads, 0, st>>>(tens, tile_begin, T, scales, partials); break;
-        default: return cudaErrorInvalidValue;
-    }
+int pick_tile_shift(long long scored_elems, int max_ctas) {
+    int shift = kMaxTileShift;
+    while (shift > kMinTileShift && (scored_elems >> shift) < 48LL * max_ctas) --shift;
+    return shift;
+}
+
+template <int FMASK, int RB>
+static cudaError_t launch_score_inst(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                                     int tile_shift, int max_ctas, const float* scales, double* partials,
+                                     LaunchStatus* status, cudaStream_t st) {
+    constexpr int smem = Ring<RB>::kSmemBytes;
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<FMASK, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)(ntiles < (long long)max_ctas ? ntiles : (long long)max_ctas);
+    score_kernel<FMASK, RB><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift, scales,
+                                                               partials, status);
     return cudaGetLastError();
 }
 
+template <int RB>
+static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                                   int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
+                                   LaunchStatus* status, cudaStream_t st) {
+    if (ntiles <= 0) return cudaSuccess;
+    if (max_ctas < 1 || tile_shift < kMinTileShift || tile_shift > kMaxTileShift) return cudaErrorInvalidValue;
+    switch (fmask) {
+        case 1: return launch_score_inst<1, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 2: return launch_score_inst<2, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 3: return launch_score_inst<3, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
-                         int fmask, const float* scales, double* partials, cudaStream_t st) {
+                         int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
+                         LaunchStatus* status, cudaStream_t st) {
     switch (rb) {
-        case 1: return launch_score_rb<1>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
-        case 2: return launch_score_rb<2>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
-        case 3: return launch_score_rb<3>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
-        case 4: return launch_score_rb<4>(tens, tile_begin, T, ntiles, fmask, scales, partials, st);
+        case 1: return launch_score_rb<1>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 2: return launch_score_rb<2>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 3: return launch_score_rb<3>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 4: return launch_score_rb<4>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
         default: return cudaErrorInvalidValue;
     }
 }

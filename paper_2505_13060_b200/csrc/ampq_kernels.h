@@ -21,8 +21,14 @@ cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, 
 cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
                           LaunchStatus* status, cudaStream_t st);
 // One launch per sample-group size rb = 1..kMaxRB, each with its own tile table.
+// Tiles hold 2^tile_shift elements; the persistent grid has at most max_ctas CTAs
+// (two per SM is the intended residency).
 cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
-                         int fmask, const float* scales, double* partials, cudaStream_t st);
+                         int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
+                         LaunchStatus* status, cudaStream_t st);
+// Largest tile shift in [kMinTileShift, kMaxTileShift] that still gives a grid of
+// max_ctas CTAs a few dozen tiles each (or the smallest shift when even that does not).
+int pick_tile_shift(long long scored_elems, int max_ctas);
 cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const double* partials, double* seg_out,
                             cudaStream_t st);
 cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParams& prm, const double* seg_out,

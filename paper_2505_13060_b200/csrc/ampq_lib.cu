@@ -106,6 +106,8 @@ struct ampq_ctx {
     bool scored = false;   // a score has been issued
     bool pending = false;  // its results have not been synchronised yet
     int launches = 0;
+    int max_ctas = 2;      // persistent scoring grid: two CTAs per SM
+    int tile_shift = kMaxTileShift;  // log2 of the scoring tile of the last score
     std::string err;
 
     // tables of the last score (host copies)
@@ -181,6 +183,14 @@ int build_tables(ampq_ctx* ctx) {
     for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
     long long tiles[kMaxRB] = {0, 0, 0, 0}, atiles = 0, slots = 0;
     int out_off = 0;
+    long long scored_elems = 0;  // value elements the scoring launches walk (shared values once per sample group)
+    for (const auto& l : ctx->layers) {
+        if (!layer_ready(l)) continue;
+        for (int k = 0; k < 2; ++k)
+            scored_elems += l.op[k].per_sample ? l.op[k].numel : l.op[k].numel * ((l.R + kMaxRB - 1) / kMaxRB);
+    }
+    ctx->tile_shift = pick_tile_shift(scored_elems, ctx->max_ctas);
+    const long long tile_elems = 1LL << ctx->tile_shift;
     for (size_t li = 0; li < ctx->layers.size(); ++li) {
         LayerRec& l = ctx->layers[li];
         if (!layer_ready(l)) continue;
@@ -218,7 +228,9 @@ int build_tables(ampq_ctx* ctx) {
             t.R = l.R;
             t.per_sample = o.per_sample;
             t.dtype = o.dtype;
-            t.tiles_per_seg = (int)((ext + kTileElems - 1) / kTileElems);
+            if ((ext + tile_elems - 1) / tile_elems > 0x7FFFFFFFLL)
+                return fail(ctx, AMPQ_ERR_TOO_LARGE, "an operand has more than 2^31-1 tiles per sample");
+            t.tiles_per_seg = (int)((ext + tile_elems - 1) / tile_elems);
             t.rgroups = o.per_sample ? 1 : (l.R + kMaxRB - 1) / kMaxRB;
             t.partial_base = slots;
             t.seg_base = (int)ctx->segs.size();
@@ -336,6 +348,8 @@ int sync_results(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
         ctx->pending = false;
     }
+    if (!ctx->tens.empty() && ctx->h_status.p->timeout)
+        return fail(ctx, AMPQ_ERR_TIMEOUT, "a bounded wait inside the scoring kernel ran out; the results of this score are invalid");
     return AMPQ_OK;
 }
 
@@ -392,6 +406,7 @@ const char* ampq_strerror(int status) {
         case AMPQ_ERR_INFEASIBLE: return "no assignment meets the budget";
         case AMPQ_ERR_TOO_LARGE: return "problem too large";
         case AMPQ_ERR_NOMEM: return "out of memory";
+        case AMPQ_ERR_TIMEOUT: return "a device-side wait timed out";
         default: return "unknown status";
     }
 }
@@ -410,6 +425,12 @@ int ampq_create(ampq_ctx** out, int device, void* cuda_stream) {
     ctx->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     DeviceGuard g(device);
     if (!g.ok || cudaFree(nullptr) != cudaSuccess) { delete ctx; return AMPQ_ERR_CUDA; }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) {
+        delete ctx;
+        return AMPQ_ERR_CUDA;
+    }
+    ctx->max_ctas = 2 * sms;
     *out = ctx;
     return AMPQ_OK;
 }
@@ -540,7 +561,7 @@ int ampq_score(ampq_ctx* ctx) {
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         for (int c = 0; c < kMaxRB; ++c) {
             if (ctx->ntiles[c] <= 0) continue;
-            AMPQ_CUDA(launch_score(c + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, st), "score");
+            AMPQ_CUDA(launch_score(c + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st), "score");
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");

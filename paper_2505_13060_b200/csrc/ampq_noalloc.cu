@@ -86,10 +86,11 @@ __global__ void noalloc_prepare_kernel(NoAllocScratch* s, const void* values, co
     s->seg_out[1] = 0.0;
 }
 
-// out = {S, D, amax}; NaN sums when the operand held Inf or NaN.
+// out = {S, D, amax}; NaN sums when the operand held Inf or NaN (or a bounded
+// wait of the scoring kernel ran out).
 __global__ void noalloc_publish_kernel(const NoAllocScratch* s, double* out) {
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
-    const bool bad = s->flag != 0;
+    const bool bad = s->flag != 0 || s->status.timeout != 0;
     const double nan = __longlong_as_double(0x7FF8000000000000LL);
     out[0] = bad ? nan : s->seg_out[0];
     out[1] = bad ? nan : s->seg_out[1];
@@ -159,7 +160,10 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     ok = ok && launch_init_amax(&s->tensor, 1, &s->amax_bits, &s->status, st) == cudaSuccess;
     ok = ok && launch_amax(&s->tensor, s->amax_tile_begin, 1, namax, &s->amax_bits, st) == cudaSuccess;
     ok = ok && launch_scales(1, fmask, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
-    ok = ok && launch_score(1, &s->tensor, s->tile_begin, 1, ntiles, fmask, s->scales, s->partials, st) == cudaSuccess;
+    int sms = 0;
+    ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
+    ok = ok && launch_score(1, &s->tensor, s->tile_begin, 1, ntiles, kMaxTileShift, 2 * sms, fmask, s->scales,
+                            s->partials, &s->status, st) == cudaSuccess;
     ok = ok && launch_finalize(&s->segment, 1, kNoAllocAcc, s->partials, s->seg_out, st) == cudaSuccess;
     if (ok) {
         noalloc_publish_kernel<<<1, 32, 0, st>>>(s, dev_out);
