@@ -14,7 +14,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libampq.so")
+# AMPQ_LIBRARY names another build of the same library (a debug or tuning build)
+LIB_PATH = os.environ.get("AMPQ_LIBRARY") or os.path.join(_HERE, "libampq.so")
 
 F32, BF16 = 0, 1
 FMT_BASE, FMT_E4M3, FMT_E5M2 = 0, 1, 2

@@ -12,8 +12,12 @@ namespace ampq {
 constexpr int kThreads = 256;          // threads per CTA of the amax kernel
 constexpr int kConsumers = 256;        // scoring threads of a scoring CTA (warps 0..7)
 constexpr int kScoreThreads = kConsumers + 32;  // plus the producer warp that feeds the shared-memory ring
+#ifndef AMPQ_SCORE_CTAS_PER_SM
+#define AMPQ_SCORE_CTAS_PER_SM 2
+#endif
+constexpr int kScoreCtasPerSm = AMPQ_SCORE_CTAS_PER_SM;  // resident scoring CTAs per SM; the persistent grid is this many per SM
 constexpr int kSubElems = 32768;       // direct path: elements between two flushes of the fp32 accumulators into fp64
-constexpr int kFlushChunks = 8;        // ring path: chunks between two flushes (at most 64 terms per fp32 lane)
+constexpr int kFlushTerms = 64;        // ring path: terms an fp32 accumulator lane takes between two flushes into fp64
 constexpr unsigned kSpinLimit = 1u << 22;  // polls of an mbarrier before a wait gives up
 // A scoring tile (one partial sum per sample and accumulator) holds 2^shift
 // elements of a segment; the host picks the shift per score so that small
@@ -26,6 +30,7 @@ static_assert((1 << kMinTileShift) % kSubElems == 0, "a scoring tile is a whole 
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
 constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
+constexpr int kScoreClasses = 2 * kMaxRB;  // scoring launches of one score: element type x samples per read
 
 // internal low-precision slots: bit 0 = E4M3, bit 1 = E5M2.  With both present
 // slot 0 is E4M3 and slot 1 is E5M2; with one present it is slot 0.

@@ -340,16 +340,18 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long* b) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* b, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* b, unsigned parity) {
+// One poll of a phase; the hardware may park the thread for up to `hint_ns`
+// before it answers, which keeps a waiting warp out of the issue slots.
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* b, unsigned parity, unsigned hint_ns = 2000u) {
     unsigned ok;
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_u32(b)), "r"(parity)
+        : "r"(smem_u32(b)), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
@@ -373,17 +375,30 @@ __device__ __forceinline__ void consumer_barrier() {  // the kConsumers scoring 
 }
 
 // Waits for a phase of an mbarrier, at most kSpinLimit polls.  A wait that runs
-// out raises the CTA's abort flag; once that is up every wait returns false at
-// once, so that all threads still walk the same control flow to the end.
+// out raises the CTA's abort flag; once that is up every wait returns false
+// after one poll, so that all threads still walk the same control flow to the
+// end.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* b, unsigned parity, volatile int* s_abort) {
-    if (*s_abort) return false;
+    if (mbar_try_wait(b, parity)) return true;
     for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+        if (*s_abort) return false;
         if (mbar_try_wait(b, parity)) return true;
-        if ((spin & 255u) == 255u && *s_abort) return false;
     }
     *s_abort = 1;
     return false;
 }
+
+// Position in the ring: stage index and the parity of the lap it is in.
+template <int STAGES>
+struct RingPos {
+    unsigned stage = 0, parity = 0;
+    __device__ __forceinline__ void advance() {
+        if (++stage == STAGES) {
+            stage = 0;
+            parity ^= 1u;
+        }
+    }
+};
 
 // CTA-wide sum of RB*NACC values in a fixed order over the scoring warps;
 // thread a < RB*NACC writes partial (r, a) of the tile.  s_red holds one
@@ -450,18 +465,83 @@ __device__ __forceinline__ void score_direct(const char* vbase, const char* cons
     }
 }
 
-// Geometry of the ring for RB gradient streams per value stream.
+// Geometry of the ring for RB gradient streams per value stream.  The
+// compile-time knobs exist for tuning builds; the defaults are what was
+// measured best on B200.
+#ifndef AMPQ_RING_U12
+#define AMPQ_RING_U12 2   // 16-byte vectors per thread, stream and chunk, RB <= 2
+#endif
+#ifndef AMPQ_RING_U34
+#define AMPQ_RING_U34 1   // the same for RB >= 3
+#endif
+#ifndef AMPQ_RING_BYTES
+#define AMPQ_RING_BYTES (64 * 1024)  // ring budget per CTA; deeper rings measured no faster
+#endif
 template <int RB>
 struct Ring {
-    static constexpr int kU = RB <= 2 ? 2 : 1;                       // 16-byte vectors per thread, stream and chunk
+    static constexpr int kU = RB <= 2 ? AMPQ_RING_U12 : AMPQ_RING_U34;
     static constexpr int kChunkBytes = kU * kConsumers * 16;          // bytes of one stream in one stage
     static constexpr int kStageBytes = (1 + RB) * kChunkBytes;
-    static constexpr int kStages = RB == 1 ? 6 : (RB == 2 ? 4 : (RB == 3 ? 6 : 4));
+#if defined(AMPQ_STAGES_RB1) && defined(AMPQ_STAGES_RB2)
+    static constexpr int kStages = RB == 1 ? AMPQ_STAGES_RB1 : (RB == 2 ? AMPQ_STAGES_RB2 : AMPQ_RING_BYTES / kStageBytes);
+#else
+    static constexpr int kStages = AMPQ_RING_BYTES / kStageBytes;
+#endif
+    static_assert(kStages >= 2, "the ring needs at least two stages");
     static constexpr int kRingBytes = kStages * kStageBytes;
     static constexpr int kRedDoubles = 2 * (kConsumers / 32) * RB * kMaxAcc;
     // ring | full[kStages] empty[kStages] | reduction blocks | abort flag
     static constexpr int kSmemBytes = kRingBytes + 2 * kStages * 8 + kRedDoubles * 8 + 16;
 };
+
+// The scoring warps' side of the ring for one tile: nchunks stages, each
+// taken into registers, handed back, then scored.
+template <int DT, int FMASK, int RB>
+__device__ __forceinline__ void consume_chunks(int nchunks, const unsigned char* ring, unsigned long long* full,
+                                               unsigned long long* empty, RingPos<Ring<RB>::kStages>& pos,
+                                               volatile int* s_abort, const float2 (&inv2)[2],
+                                               const float2 (&nsc2)[2], Acc<Fm<FMASK>::kAcc> (&acc)[RB],
+                                               double (&acc64)[RB][Fm<FMASK>::kAcc]) {
+    using RG = Ring<RB>;
+    using E = Elem<DT>;
+    constexpr int NACC = Fm<FMASK>::kAcc;
+    constexpr int U = RG::kU;
+    constexpr int NP = E::kPerVec / 2;
+    const int tid = threadIdx.x;
+    int since_flush = 0;
+    for (int c = 0; c < nchunks; ++c) {
+        const bool ok = mbar_wait(full + pos.stage, pos.parity, s_abort);
+        uint4 v[U], g[RB][U];
+        if (ok) {
+            const unsigned char* st = ring + pos.stage * RG::kStageBytes + tid * 16;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                v[u] = lds_v4(st + u * kConsumers * 16);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) g[r][u] = lds_v4(st + (1 + r) * RG::kChunkBytes + u * kConsumers * 16);
+            }
+        }
+        __syncwarp();
+        if (ok && (tid & 31) == 0) mbar_arrive(empty + pos.stage);  // the warp's vectors are in registers
+        pos.advance();
+        if (ok) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float2 z[NP], gg[RB][NP];
+                E::unpack(v[u], z);
+#pragma unroll
+                for (int r = 0; r < RB; ++r) E::unpack(g[r][u], gg[r]);
+                accumulate_pairs<FMASK, RB, NP>(z, gg, inv2, nsc2, acc);
+            }
+        }
+        // at most kFlushTerms terms per fp32 lane between two flushes
+        since_flush += U * NP;
+        if (since_flush >= kFlushTerms) {
+            flush_acc<NACC, RB>(acc, acc64);
+            since_flush = 0;
+        }
+    }
+}
 
 // Where a tile lives.
 struct TileGeom {
@@ -502,20 +582,19 @@ __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, i
 // the bytes in flight do not depend on how long the arithmetic of a chunk
 // takes.  A scoring thread takes its 16-byte vectors of a stage into
 // registers, hands the stage back and then does the arithmetic.  fp32 sums are
-// flushed into fp64 every kFlushChunks chunks; a tile ends with the CTA-wide
+// flushed into fp64 every kFlushTerms terms; a tile ends with the CTA-wide
 // ordered sum and one partial per (sample, accumulator).
 //
-// One launch per sample-group size RB (1..4): per-sample operands and the
-// single-sample remainder of shared operands run with RB = 1; shared operands
-// (weights) are read once per group of up to four samples.
-template <int FMASK, int RB>
-__global__ void __launch_bounds__(kScoreThreads, 2)
+// One launch per element type DT and sample-group size RB (1..4): per-sample
+// operands and the single-sample remainder of shared operands run with RB = 1;
+// shared operands (weights) are read once per group of up to four samples.
+template <int DT, int FMASK, int RB>
+__global__ void __launch_bounds__(kScoreThreads, kScoreCtasPerSm)
 score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
              int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
              LaunchStatus* __restrict__ status) {
     using RG = Ring<RB>;
     constexpr int NACC = Fm<FMASK>::kAcc;
-    constexpr int U = RG::kU;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* ring = smem;
     unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + RG::kRingBytes);
@@ -534,7 +613,8 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
     __syncthreads();
 
     const bool producer = threadIdx.x >= kConsumers;
-    unsigned it = 0;  // chunks through the ring so far (same count on both sides)
+    unsigned it = 0;  // chunks the producer has put into the ring so far
+    RingPos<RG::kStages> pos;  // both sides walk the ring in the same order
     int t = 0;        // tensor of the current tile; tiles only move forward
     if (producer) {
         if (threadIdx.x == kConsumers) {
@@ -542,7 +622,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
                 while (tile >= __ldg(tile_begin + t + 1)) ++t;
                 const Tensor& tn = tens[t];
                 const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
-                const int es = tn.dtype == 0 ? 4 : 2;
+                constexpr int es = Elem<DT>::kBytes;
                 const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
                 const char* gb[RB];
                 bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
@@ -552,16 +632,18 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
                     aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
                 }
                 const int nchunks = aligned ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
-                for (int c = 0; c < nchunks; ++c, ++it) {
-                    const unsigned s = it % RG::kStages, lap = it / RG::kStages;
-                    if (lap > 0 && !mbar_wait(empty + s, (lap - 1) & 1, s_abort)) break;
-                    unsigned char* dst = ring + s * RG::kStageBytes;
-                    mbar_arrive_expect_tx(full + s, RG::kStageBytes);
-                    bulk_load(dst, vb + (long long)c * RG::kChunkBytes, RG::kChunkBytes, full + s);
+                for (int c = 0; c < nchunks; ++c) {
+                    // the stage must have been handed back once per earlier lap
+                    if (it >= (unsigned)RG::kStages && !mbar_wait(empty + pos.stage, pos.parity ^ 1u, s_abort)) break;
+                    unsigned char* dst = ring + pos.stage * RG::kStageBytes;
+                    mbar_arrive_expect_tx(full + pos.stage, RG::kStageBytes);
+                    bulk_load(dst, vb + (long long)c * RG::kChunkBytes, RG::kChunkBytes, full + pos.stage);
 #pragma unroll
                     for (int r = 0; r < RB; ++r)
                         bulk_load(dst + (1 + r) * RG::kChunkBytes, gb[r] + (long long)c * RG::kChunkBytes,
-                                  RG::kChunkBytes, full + s);
+                                  RG::kChunkBytes, full + pos.stage);
+                    pos.advance();
+                    ++it;
                 }
                 if (*s_abort) break;
             }
@@ -581,13 +663,12 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
     }
 
     // ---- scoring warps
-    const int tid = threadIdx.x;
     int red_block = 0;
     for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         while (tile >= __ldg(tile_begin + t + 1)) ++t;
         const Tensor& tn = tens[t];
         const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
-        const int es = tn.dtype == 0 ? 4 : 2;
+        constexpr int es = Elem<DT>::kBytes;
         float2 inv2[2], nsc2[2];
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
@@ -615,45 +696,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
                 acc64[r][a] = 0.0;
                 acc[r].v[a] = make_float2(0.0f, 0.0f);
             }
-        for (int c = 0; c < nchunks; ++c, ++it) {
-            const unsigned s = it % RG::kStages, lap = it / RG::kStages;
-            const bool ok = mbar_wait(full + s, lap & 1, s_abort);
-            uint4 v[U], g[RB][U];
-            if (ok) {
-                const unsigned char* st = ring + s * RG::kStageBytes;
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    v[u] = lds_v4(st + (u * kConsumers + tid) * 16);
-#pragma unroll
-                    for (int r = 0; r < RB; ++r)
-                        g[r][u] = lds_v4(st + (1 + r) * RG::kChunkBytes + (u * kConsumers + tid) * 16);
-                }
-            }
-            __syncwarp();
-            if (ok && (tid & 31) == 0) mbar_arrive(empty + s);  // the warp's vectors are in registers
-            if (ok) {
-                if (tn.dtype == 0) {
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        float2 z[2], gg[RB][2];
-                        Elem<0>::unpack(v[u], z);
-#pragma unroll
-                        for (int r = 0; r < RB; ++r) Elem<0>::unpack(g[r][u], gg[r]);
-                        accumulate_pairs<FMASK, RB, 2>(z, gg, inv2, nsc2, acc);
-                    }
-                } else {
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        float2 z[4], gg[RB][4];
-                        Elem<1>::unpack(v[u], z);
-#pragma unroll
-                        for (int r = 0; r < RB; ++r) Elem<1>::unpack(g[r][u], gg[r]);
-                        accumulate_pairs<FMASK, RB, 4>(z, gg, inv2, nsc2, acc);
-                    }
-                }
-            }
-            if ((c % kFlushChunks) == kFlushChunks - 1) flush_acc<NACC, RB>(acc, acc64);
-        }
+        consume_chunks<DT, FMASK, RB>(nchunks, ring, full, empty, pos, s_abort, inv2, nsc2, acc, acc64);
         flush_acc<NACC, RB>(acc, acc64);
         // what the ring did not carry
         const int done = (int)(((long long)nchunks * RG::kChunkBytes) / es);
@@ -661,10 +704,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
             const char* gt[RB];
 #pragma unroll
             for (int r = 0; r < RB; ++r) gt[r] = gb[r] + (long long)done * es;
-            if (tn.dtype == 0)
-                score_direct<0, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
-            else
-                score_direct<1, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
+            score_direct<DT, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
         }
         reduce_and_store<NACC, RB>(acc64, s_red + red_block * (kConsumers / 32) * RB * NACC, partials, q.slot0,
                                    tn.tiles_per_seg);
@@ -776,43 +816,54 @@ int pick_tile_shift(long long scored_elems, int max_ctas) {
     return shift;
 }
 
-template <int FMASK, int RB>
+template <int DT, int FMASK, int RB>
 static cudaError_t launch_score_inst(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                      int tile_shift, int max_ctas, const float* scales, double* partials,
                                      LaunchStatus* status, cudaStream_t st) {
     constexpr int smem = Ring<RB>::kSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<FMASK, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(ntiles < (long long)max_ctas ? ntiles : (long long)max_ctas);
-    score_kernel<FMASK, RB><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift, scales,
-                                                               partials, status);
+    score_kernel<DT, FMASK, RB><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift, scales,
+                                                                   partials, status);
     return cudaGetLastError();
 }
 
-template <int RB>
+template <int DT, int RB>
 static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                    int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
                                    LaunchStatus* status, cudaStream_t st) {
-    if (ntiles <= 0) return cudaSuccess;
-    if (max_ctas < 1 || tile_shift < kMinTileShift || tile_shift > kMaxTileShift) return cudaErrorInvalidValue;
     switch (fmask) {
-        case 1: return launch_score_inst<1, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 2: return launch_score_inst<2, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 3: return launch_score_inst<3, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 1: return launch_score_inst<DT, 1, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 2: return launch_score_inst<DT, 2, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 3: return launch_score_inst<DT, 3, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
         default: return cudaErrorInvalidValue;
     }
 }
 
-cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
-                         int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                         LaunchStatus* status, cudaStream_t st) {
+template <int DT>
+static cudaError_t launch_score_dt(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                                   int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
+                                   LaunchStatus* status, cudaStream_t st) {
     switch (rb) {
-        case 1: return launch_score_rb<1>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 2: return launch_score_rb<2>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 3: return launch_score_rb<3>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 4: return launch_score_rb<4>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 1: return launch_score_rb<DT, 1>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 2: return launch_score_rb<DT, 2>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 3: return launch_score_rb<DT, 3>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 4: return launch_score_rb<DT, 4>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
         default: return cudaErrorInvalidValue;
     }
+}
+
+cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+                         int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
+                         LaunchStatus* status, cudaStream_t st) {
+    if (ntiles <= 0) return cudaSuccess;
+    if (max_ctas < 1 || tile_shift < kMinTileShift || tile_shift > kMaxTileShift) return cudaErrorInvalidValue;
+    if (dtype == 0)
+        return launch_score_dt<0>(rb, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+    if (dtype == 1)
+        return launch_score_dt<1>(rb, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const double* partials, double* seg_out,

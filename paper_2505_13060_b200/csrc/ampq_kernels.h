@@ -20,10 +20,11 @@ cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, 
                         unsigned* amax_bits, cudaStream_t st);
 cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
                           LaunchStatus* status, cudaStream_t st);
-// One launch per sample-group size rb = 1..kMaxRB, each with its own tile table.
+// One launch per element type (0 = fp32, 1 = bf16) and sample-group size rb =
+// 1..kMaxRB, each with its own tile table.
 // Tiles hold 2^tile_shift elements; the persistent grid has at most max_ctas CTAs
 // (two per SM is the intended residency).
-cudaError_t launch_score(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                          int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
                          LaunchStatus* status, cudaStream_t st);
 // Largest tile shift in [kMinTileShift, kMaxTileShift] that still gives a grid of

@@ -106,21 +106,22 @@ struct ampq_ctx {
     bool scored = false;   // a score has been issued
     bool pending = false;  // its results have not been synchronised yet
     int launches = 0;
-    int max_ctas = 2;      // persistent scoring grid: two CTAs per SM
+    int max_ctas = kScoreCtasPerSm;  // persistent scoring grid: kScoreCtasPerSm CTAs per SM
     int tile_shift = kMaxTileShift;  // log2 of the scoring tile of the last score
     std::string err;
 
     // tables of the last score (host copies)
     std::vector<Tensor> tens;
-    std::vector<long long> tile_begin[kMaxRB], amax_tile_begin;  // tile_begin[rb-1]: tiles scored with rb samples
+    // tile_begin[dtype * kMaxRB + rb - 1]: tiles of `dtype` operands scored with rb samples per read
+    std::vector<long long> tile_begin[kScoreClasses], amax_tile_begin;
     std::vector<Segment> segs;
     std::vector<Layer> lay;
     std::vector<int> scored_layer_ids;
-    long long ntiles[kMaxRB] = {0, 0, 0, 0}, namax_tiles = 0, nslots = 0;
+    long long ntiles[kScoreClasses] = {}, namax_tiles = 0, nslots = 0;
     int layer_out_doubles = 0;
 
     DevBuf<Tensor> d_tens;
-    DevBuf<long long> d_tile_begin[kMaxRB], d_amax_tile_begin;
+    DevBuf<long long> d_tile_begin[kScoreClasses], d_amax_tile_begin;
     DevBuf<Segment> d_segs;
     DevBuf<Layer> d_lay;
     DevBuf<unsigned> d_amax_bits;
@@ -181,7 +182,7 @@ int build_tables(ampq_ctx* ctx) {
     for (auto& tb : ctx->tile_begin) tb.clear();
     ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
     for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
-    long long tiles[kMaxRB] = {0, 0, 0, 0}, atiles = 0, slots = 0;
+    long long tiles[kScoreClasses] = {}, atiles = 0, slots = 0;
     int out_off = 0;
     long long scored_elems = 0;  // value elements the scoring launches walk (shared values once per sample group)
     for (const auto& l : ctx->layers) {
@@ -238,15 +239,16 @@ int build_tables(ampq_ctx* ctx) {
             // per-sample operands: one single-sample tile per (sample, value tile);
             // shared operands: value tiles x full groups of kMaxRB samples, plus one
             // remainder group of R mod kMaxRB samples
-            long long my_tiles[kMaxRB] = {0, 0, 0, 0};
+            long long my_tiles[kScoreClasses] = {};
+            const int c0 = (o.dtype == AMPQ_F32 ? 0 : 1) * kMaxRB;  // classes of this operand's dtype
             if (o.per_sample) {
-                my_tiles[0] = (long long)l.R * t.tiles_per_seg;
+                my_tiles[c0] = (long long)l.R * t.tiles_per_seg;
             } else {
-                my_tiles[kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
-                if (l.R % kMaxRB) my_tiles[l.R % kMaxRB - 1] += t.tiles_per_seg;
+                my_tiles[c0 + kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
+                if (l.R % kMaxRB) my_tiles[c0 + l.R % kMaxRB - 1] += t.tiles_per_seg;
             }
             const long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
-            for (int c = 0; c < kMaxRB; ++c) {
+            for (int c = 0; c < kScoreClasses; ++c) {
                 ctx->tile_begin[c].push_back(tiles[c]);
                 tiles[c] += my_tiles[c];
             }
@@ -269,7 +271,7 @@ int build_tables(ampq_ctx* ctx) {
         ctx->scored_layer_ids.push_back((int)li);
     }
     long long most = atiles;
-    for (int c = 0; c < kMaxRB; ++c) {
+    for (int c = 0; c < kScoreClasses; ++c) {
         ctx->tile_begin[c].push_back(tiles[c]);
         ctx->ntiles[c] = tiles[c];
         if (tiles[c] > most) most = tiles[c];
@@ -287,7 +289,7 @@ int upload_tables(ampq_ctx* ctx) {
     const size_t T = ctx->tens.size(), L = ctx->lay.size(), S = ctx->segs.size();
     const int nacc = 1 + (ctx->F - 1);
     AMPQ_CUDA(ctx->d_tens.ensure(T), "cudaMalloc(tensors)");
-    for (int c = 0; c < kMaxRB; ++c) AMPQ_CUDA(ctx->d_tile_begin[c].ensure(T + 1), "cudaMalloc(tile_begin)");
+    for (int c = 0; c < kScoreClasses; ++c) AMPQ_CUDA(ctx->d_tile_begin[c].ensure(T + 1), "cudaMalloc(tile_begin)");
     AMPQ_CUDA(ctx->d_amax_tile_begin.ensure(T + 1), "cudaMalloc(amax_tile_begin)");
     AMPQ_CUDA(ctx->d_segs.ensure(S), "cudaMalloc(segments)");
     AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
@@ -309,7 +311,7 @@ int upload_tables(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tens.p, ctx->tens.data(), T * sizeof(Tensor), cudaMemcpyHostToDevice, st), "H2D tensors");
         AMPQ_CUDA(cudaMemsetAsync(ctx->d_scales.p, 0, T * 2 * kMaxLow * sizeof(float), st), "memset scales");
     }
-    for (int c = 0; c < kMaxRB; ++c)
+    for (int c = 0; c < kScoreClasses; ++c)
         AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tile_begin[c].p, ctx->tile_begin[c].data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D tile_begin");
     AMPQ_CUDA(cudaMemcpyAsync(ctx->d_amax_tile_begin.p, ctx->amax_tile_begin.data(), (T + 1) * sizeof(long long), cudaMemcpyHostToDevice, st), "H2D amax_tile_begin");
     if (S) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_segs.p, ctx->segs.data(), S * sizeof(Segment), cudaMemcpyHostToDevice, st), "H2D segments");
@@ -430,7 +432,7 @@ int ampq_create(ampq_ctx** out, int device, void* cuda_stream) {
         delete ctx;
         return AMPQ_ERR_CUDA;
     }
-    ctx->max_ctas = 2 * sms;
+    ctx->max_ctas = kScoreCtasPerSm * sms;
     *out = ctx;
     return AMPQ_OK;
 }
@@ -559,9 +561,9 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st), "scales");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
-        for (int c = 0; c < kMaxRB; ++c) {
+        for (int c = 0; c < kScoreClasses; ++c) {
             if (ctx->ntiles[c] <= 0) continue;
-            AMPQ_CUDA(launch_score(c + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st), "score");
+            AMPQ_CUDA(launch_score(c / kMaxRB, c % kMaxRB + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st), "score");
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");

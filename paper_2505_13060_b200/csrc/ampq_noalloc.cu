@@ -162,7 +162,7 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     ok = ok && launch_scales(1, fmask, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
     int sms = 0;
     ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
-    ok = ok && launch_score(1, &s->tensor, s->tile_begin, 1, ntiles, kMaxTileShift, 2 * sms, fmask, s->scales,
+    ok = ok && launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &s->tensor, s->tile_begin, 1, ntiles, kMaxTileShift, kScoreCtasPerSm * sms, fmask, s->scales,
                             s->partials, &s->status, st) == cudaSuccess;
     ok = ok && launch_finalize(&s->segment, 1, kNoAllocAcc, s->partials, s->seg_out, st) == cudaSuccess;
     if (ok) {
