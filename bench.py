@@ -36,6 +36,17 @@ METRIC = "sensitivity_pass_throughput_scored"
 UNIT = "GB/s"
 NUM_BLOCKS = 80
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per scored byte of the
+# scoring launches, from the ncu capture summarised in
+# profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md (a 1.98 GB case;
+# traffic grows in proportion to the elements).  It holds only for the kernel
+# source it was taken on: `kernels_sha256` is the digest of ampq_kernels.cu +
+# ampq_device.h at capture time, and the bench reports traffic = null otherwise.
+NCU_TRAFFIC = {
+    "kernels_sha256": "32204b95bb211665fe84ccb89aa98cce9e295016f1e858ba6e71f985ae329f32",
+    "dram_bytes_per_scored_byte": {"e4m3": 1.0048},
+    "source": "profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md",
+}
 
 
 def parse_args():
@@ -68,6 +79,16 @@ def hbm_peak():
         except Exception:
             pass
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernels_digest() -> str:
+    import hashlib
+
+    h = hashlib.sha256()
+    for f in ("ampq_kernels.cu", "ampq_device.h"):
+        with open(os.path.join(ROOT, "paper_2505_13060_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 
 
 # --------------------------------------------------------------------------
@@ -127,20 +148,23 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------
-def oracle_sample(threads: int, low_fmts, device):
-    """The oracle's bounded sample: the q, k, v, o linear layers of one
-    70B-shaped block (all R = 2 samples; 2.28 GB of scored bytes).  Returns
-    (host tensors per layer, scored bytes, description)."""
+def oracle_sample(threads: int, low_fmts, device, whole_block: bool):
+    """The oracle's bounded sample of the 70B-shaped workload: one whole block
+    (7 linear layers, R = 2 samples; 7.68 GB of scored bytes, about 10 s on 16
+    cores) or only its q, k, v, o layers (1.98 GB; the per-step sample of the
+    reference arm, which repeats it `--steps` times).  Returns (host tensors per
+    layer, scored bytes, description)."""
     from paper_2505_13060_b200 import synth
 
-    specs = synth.llama70b_block()[:4]
+    specs = synth.llama70b_block() if whole_block else synth.llama70b_block()[:4]
     layers, nbytes = [], 0
     for i, s in enumerate(specs):
         lt = synth.make_layer(s, device, seed=1234, layer=i)
         layers.append((s, [synth.to_numpy(t) for t in lt.values], [synth.to_numpy(t) for t in lt.grads]))
         nbytes += s.scored_bytes()
         del lt
-    return layers, nbytes, "q,k,v,o linear layers of one Llama-70B-shaped block (R=2 x 4096 tokens, bf16)"
+    what = "all 7 linear layers" if whole_block else "q,k,v,o linear layers"
+    return layers, nbytes, what + " of one Llama-70B-shaped block (R=2 x 4096 tokens, bf16)"
 
 
 def time_oracle(layers, threads: int, low_fmts):
@@ -193,7 +217,7 @@ def run_reference(args):
     low = {"e4m3": [1], "e5m2": [2], "both": [1, 2]}[args.formats]
     threads = args.cpu_threads or usable_cores()
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    layers, nbytes, desc = oracle_sample(threads, low, dev)
+    layers, nbytes, desc = oracle_sample(threads, low, dev, whole_block=False)
     for _ in range(max(0, min(args.warmup, 1))):  # a warm-up pass of a deterministic CPU loop buys nothing more
         time_oracle(layers, threads, low)
     times = []
@@ -217,6 +241,42 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------
+def workload_specs(workload: str, layers: str = ""):
+    """Layer specs of one block of the named workload (optionally a subset of its layers)."""
+    from paper_2505_13060_b200 import synth
+
+    specs = synth.llama70b_block() if workload == "llama70b" else synth.llama7b_block()
+    if layers:
+        keep = layers.split(",")
+        specs = [sp for sp in specs if sp.name in keep]
+        if not specs:
+            raise SystemExit("--layers matched no layer of the block")
+    return specs
+
+
+def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int):
+    """Registers `blocks` blocks of `specs` in ctx.  Block b is bound to device
+    slot b mod nres; each slot is a full block of distinct random tensors.
+    Returns (slots, layer ids, scored bytes of one score)."""
+    import torch
+
+    from paper_2505_13060_b200 import binding as ampq
+    from paper_2505_13060_b200 import synth
+
+    slots = []
+    for s in range(nres):
+        slots.append([synth.make_layer(sp, dev, seed=seed, layer=len(specs) * s + i) for i, sp in enumerate(specs)])
+    torch.cuda.synchronize()
+    ids, scored_bytes = [], 0
+    for b in range(blocks):
+        for i, sp in enumerate(specs):
+            lid = ctx.register_layer(sp.kind, "blk%d.%s" % (b, sp.name), sp.R)
+            ampq.bind_layer_tensors(ctx, lid, slots[b % nres][i])
+            ids.append(lid)
+            scored_bytes += sp.scored_bytes()
+    return slots, ids, scored_bytes
+
+
 def run_b200(args):
     import torch
 
@@ -238,30 +298,13 @@ def run_b200(args):
     dev = torch.device("cuda", local_rank)
     fmts = {"e4m3": [0, 1], "e5m2": [0, 2], "both": [0, 1, 2]}[args.formats]
 
-    # ---- resident slots: full 70B-shaped blocks of distinct random tensors
-    specs = synth.llama70b_block() if args.workload == "llama70b" else synth.llama7b_block()
-    if args.layers:
-        keep = args.layers.split(",")
-        specs = [sp for sp in specs if sp.name in keep]
-        if not specs:
-            raise SystemExit("--layers matched no layer of the block")
+    specs = workload_specs(args.workload, args.layers)
     block_gb = sum(sp.scored_bytes() for sp in specs) / 1e9
     nres = max(1, min(args.resident_blocks, args.blocks))
-    slots = []
-    for s in range(nres):
-        slots.append([synth.make_layer(sp, dev, seed=100 + rank, layer=len(specs) * s + i) for i, sp in enumerate(specs)])
-    torch.cuda.synchronize()
     stream = torch.cuda.Stream(device=dev)
     ctx = ampq.Context(local_rank, stream.cuda_stream)
     ctx.set_formats(fmts)
-    ids = []
-    scored_bytes = 0
-    for b in range(args.blocks):
-        for i, sp in enumerate(specs):
-            lid = ctx.register_layer(sp.kind, "blk%d.%s" % (b, sp.name), sp.R)
-            ampq.bind_layer_tensors(ctx, lid, slots[b % nres][i])
-            ids.append(lid)
-            scored_bytes += sp.scored_bytes()
+    slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev, seed=100 + rank)
     value_bytes = args.blocks * sum(sp.value_bytes() for sp in specs)
     ctx.set_timing(True)
 
@@ -312,15 +355,10 @@ def run_b200(args):
         "amax_kernel_gbs": value_bytes / (sum(amax_ms) / len(amax_ms) * 1e-3) / 1e9,
         "frac_of_8000_datasheet": achieved / 8000.0,
     }
-    traffic_file = os.path.join(ROOT, "profiles", "score_kernel_traffic.json")
-    if os.path.exists(traffic_file):
-        try:
-            tj = json.load(open(traffic_file))
-            # DRAM bytes per scored byte from an ncu capture of a smaller case, scaled to this launch
-            roofline["traffic"] = tj["dram_bytes_per_scored_byte"][args.formats] * scored_bytes
-            roofline["traffic_source"] = tj["source"]
-        except Exception:
-            pass
+    ratio = NCU_TRAFFIC["dram_bytes_per_scored_byte"].get(args.formats)
+    if ratio is not None and kernels_digest() == NCU_TRAFFIC["kernels_sha256"]:
+        roofline["traffic"] = ratio * scored_bytes  # scaled from the small capture to this launch
+        roofline["traffic_source"] = NCU_TRAFFIC["source"]
 
     # ---- end to end: tensors in pinned host memory, one block per step
     e2e = None
@@ -366,11 +404,16 @@ def run_b200(args):
         ectx.destroy()
         del host_layers
 
+    check = {"s_mean_layer0": first["s_mean"], "d_meas_layer0": float(first["d_meas"][1])}
+    ctx.destroy()
+    del slots
+    torch.cuda.empty_cache()
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only
     cpu = None
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         threads = args.cpu_threads or usable_cores()
-        layers, nbytes, desc = oracle_sample(threads, fmts[1:], dev)
+        layers, nbytes, desc = oracle_sample(threads, fmts[1:], dev, whole_block=True)
         dt, njobs, out = time_oracle(layers, threads, fmts[1:])
         cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": min(threads, njobs), "kind": "oracle",
                "sample": desc + ", %.2f GB scored in %.1f s" % (nbytes / 1e9, dt)}
@@ -390,11 +433,10 @@ def run_b200(args):
             },
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu,
-            "check": {"s_mean_layer0": first["s_mean"], "d_meas_layer0": float(first["d_meas"][1])},
+            "check": check,
             "pct_of_hbm_peak": {"measured_%.0f" % peak: 100.0 * value / peak, "datasheet_8000": 100.0 * value / 8000.0},
         }
         print(json.dumps(line), flush=True)
-    ctx.destroy()
     if dist is not None:
         dist.destroy_process_group()
 

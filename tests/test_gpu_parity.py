@@ -338,3 +338,37 @@ def test_host_bound_operands_and_determinism(ampq, orc):
         assert a["d_meas"].tobytes() == b["d_meas"].tobytes()
     hctx.destroy()
     ctx.destroy()
+
+
+def test_full_size_llama70b_sampled_layers(ampq, orc):
+    """The benchmark's own launch configuration: all 80 blocks x 7 linear layers
+    of the Llama-70B-shaped workload in one score (blocks bound to a few resident
+    slots, as bench.py binds them).  The oracle recomputes sampled layers one by
+    one -- the smallest (k), a mid-sized one (o) and the largest (down) -- and
+    every block must reproduce, bit for bit, the block that shares its slot."""
+    import bench
+
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24e9:
+        pytest.skip("needs 24 GB of free device memory")
+    specs = bench.workload_specs("llama70b")
+    nres, blocks = 2, 80
+    ctx = _ctx(ampq, (0, E4M3))
+    slots, ids, scored = bench.bind_workload(ctx, specs, blocks, nres, torch.device("cuda", 0), seed=7)
+    assert len(ids) == 560 and scored == 614717194240
+    ctx.score()
+    names = [s.name for s in specs]
+    for blk, name in ((0, "k"), (1, "o"), (1, "down")):
+        i = names.index(name)
+        lt = slots[blk % nres][i]
+        ref = oracle_layer(orc, lt, [E4M3], threads=8)
+        compare_layer(ampq, ctx, ids[7 * blk + i], ref, 2, "blk%d.%s" % (blk, name))
+        assert 0.2 * ref["d_model"][1] < ref["d_meas"][1] < 1.2 * ref["d_model"][1]
+    first = [ctx.get_layer(ids[j]) for j in range(7 * nres)]
+    for b in range(nres, blocks):
+        for i in range(7):
+            a, got = first[7 * (b % nres) + i], ctx.get_layer(ids[7 * b + i])
+            assert a["amax"].tobytes() == got["amax"].tobytes()
+            assert a["s_per_sample"].tobytes() == got["s_per_sample"].tobytes()
+            assert a["d_meas_per_sample"].tobytes() == got["d_meas_per_sample"].tobytes()
+    ctx.destroy()
