@@ -173,6 +173,12 @@ int ampq_clear_groups(ampq_ctx *ctx);
  * left fold in l, from the last score.  d_out[Pj], host pointer. */
 int ampq_group_costs(ampq_ctx *ctx, int group_id, int d_mode, double *d_out);
 
+/* The same sums from a caller-supplied per-layer table (no context, no GPU;
+ * used when layers were scored by several contexts or processes): d_layer is
+ * [L][F] row-major, layer_ids[l] in [0, L).  d_out[Pj]. */
+int ampq_group_costs_table(const int *layer_ids, int Lj, const unsigned char *Q, int Pj,
+                           const double *d_layer, int L, int F, double *d_out);
+
 /* budget = tau^2 * (1/R) sum_r losses[r]^2 (Sec. 2.1; E[g^2] is the
  * mean-square loss of Algorithm 1 step 2).  Needs no context. */
 int ampq_budget_from_tau(double tau, const double *losses, int R, double *budget);

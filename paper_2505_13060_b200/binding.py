@@ -34,6 +34,7 @@ EXPORTS = [
     "ampq_last_launch_count", "ampq_set_timing", "ampq_get_timing", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
     "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
+    "ampq_group_costs_table",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -78,6 +79,7 @@ def lib():
     L.ampq_define_group.argtypes = [vp, vp, i, vp, vp, i, ip]
     L.ampq_clear_groups.argtypes = [vp]
     L.ampq_group_costs.argtypes = [vp, i, i, vp]
+    L.ampq_group_costs_table.argtypes = [vp, i, vp, i, vp, i, i, vp]
     L.ampq_budget_from_tau.argtypes = [C.c_double, vp, i, dp]
     L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
     L.ampq_select.argtypes = [vp, i, C.c_double, vp, dp, dp]
@@ -101,6 +103,21 @@ def budget_from_tau(tau: float, losses) -> float:
     if rc:
         raise AmpqError(rc)
     return out.value
+
+
+def group_costs_table(layer_ids, Q, d_layer) -> np.ndarray:
+    """d_{j,p} of one group from a per-layer table d_layer[L, F]; Q: [Lj, Pj]."""
+    ids = np.ascontiguousarray(layer_ids, dtype=np.int32)
+    Q = np.asarray(Q, dtype=np.uint8)
+    Lj, Pj = Q.shape
+    Qf = np.ascontiguousarray(Q.T).reshape(-1)  # Q[l + Lj*p]
+    d_layer = np.ascontiguousarray(d_layer, dtype=np.float64)
+    out = np.zeros(Pj)
+    rc = lib().ampq_group_costs_table(_np_ptr(ids), Lj, _np_ptr(Qf), Pj, _np_ptr(d_layer), d_layer.shape[0],
+                                      d_layer.shape[1], _np_ptr(out))
+    if rc:
+        raise AmpqError(rc, "ampq_group_costs_table")
+    return out
 
 
 def select_tables(c_tables, d_tables, budget: float):

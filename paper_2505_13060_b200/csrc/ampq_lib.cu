@@ -732,6 +732,21 @@ int ampq_group_costs(ampq_ctx* ctx, int group_id, int d_mode, double* d_out) {
     return group_costs_impl(ctx, ctx->groups[group_id], d_mode, d_out);
 }
 
+int ampq_group_costs_table(const int* layer_ids, int Lj, const unsigned char* Q, int Pj, const double* d_layer,
+                           int L, int F, double* d_out) {
+    if (!layer_ids || !Q || !d_layer || !d_out || Lj < 1 || Pj < 1 || L < 1 || F < 1) return AMPQ_ERR_INVALID;
+    for (int l = 0; l < Lj; ++l)
+        if (layer_ids[l] < 0 || layer_ids[l] >= L) return AMPQ_ERR_INVALID;
+    for (long long i = 0; i < (long long)Lj * Pj; ++i)
+        if (Q[i] >= F) return AMPQ_ERR_INVALID;
+    for (int p = 0; p < Pj; ++p) {
+        double d = 0.0;
+        for (int l = 0; l < Lj; ++l) d += d_layer[(size_t)layer_ids[l] * F + Q[l + (size_t)Lj * p]];
+        d_out[p] = d;
+    }
+    return AMPQ_OK;
+}
+
 int ampq_budget_from_tau(double tau, const double* losses, int R, double* budget) {
     if (!losses || !budget || R < 1 || !(tau >= 0.0)) return AMPQ_ERR_INVALID;
     double a = 0.0;
