@@ -210,6 +210,32 @@ void orc_codes(int dtype, const void *values, long long n, int fmt, float inv_sc
     }
 }
 
+/* Storing an fp32 value as bf16: round to nearest, ties to even, on the upper
+ * 16 bits (finite inputs only). */
+static inline uint16_t orc_f32_to_bf16(float f) {
+    uint32_t b;
+    memcpy(&b, &f, 4);
+    uint32_t lsb = (b >> 16) & 1u;
+    b += 0x7FFFu + lsb;
+    return (uint16_t)(b >> 16);
+}
+
+/* The quantised operand itself, z^ = z + z~ (Sec. 2.2): z^_k = decode_f(q_k) * scale
+ * evaluated as one fp32 product (the exact product rounded once), then stored
+ * in the operand's own type (fp32 as is, bf16 by round-to-nearest-even).  This
+ * is what a model run "in format f" feeds to the layer. */
+void orc_fake_quant(int dtype, const void *values, long long n, int fmt, float scale,
+                    float inv_scale, void *out) {
+    for (long long k = 0; k < n; ++k) {
+        double z = (double)orc_load_f(dtype, values, k);
+        float y = (float)(z * (double)inv_scale);
+        unsigned q = orc_fp8_encode(fmt, y);
+        float zh = (float)(orc_fp8_decode(fmt, q) * (double)scale);
+        if (dtype == ORC_F32) ((float *)out)[k] = zh;
+        else ((uint16_t *)out)[k] = orc_f32_to_bf16(zh);
+    }
+}
+
 /* Steps 3-4 for one segment (one tensor, one sample): over its n elements
  *   S    = sum_k (z_k g_k)^2                     (the paper's sensitivity term)
  *   D_f  = sum_k (g_k e_k)^2,  e_k = decode_f(q_k) * scale_f - z_k

@@ -57,6 +57,8 @@ def lib():
         L.orc_scales.argtypes = [C.c_int, C.c_float, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.orc_codes.restype = None
         L.orc_codes.argtypes = [C.c_int, C.c_void_p, C.c_longlong, C.c_int, C.c_float, C.c_void_p]
+        L.orc_fake_quant.restype = None
+        L.orc_fake_quant.argtypes = [C.c_int, C.c_void_p, C.c_longlong, C.c_int, C.c_float, C.c_float, C.c_void_p]
         L.orc_score_segment.restype = None
         L.orc_score_segment.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_longlong, C.c_int,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -130,6 +132,15 @@ def codes(values: np.ndarray, fmt: int, inv_scale) -> np.ndarray:
     out = np.empty(v.size, dtype=np.uint8)
     lib().orc_codes(_dtype_of(v), _ptr(v), v.size, fmt, C.c_float(float(inv_scale)), _ptr(out))
     return out
+
+
+def fake_quant(values: np.ndarray, fmt: int, scale, inv_scale) -> np.ndarray:
+    """The quantised operand z^ = decode(q) * scale in the operand's own dtype."""
+    v = np.ascontiguousarray(values).reshape(-1)
+    out = np.empty_like(v)
+    lib().orc_fake_quant(_dtype_of(v), _ptr(v), v.size, fmt, C.c_float(float(scale)),
+                         C.c_float(float(inv_scale)), _ptr(out))
+    return out.reshape(np.shape(values))
 
 
 def score_segment(values: np.ndarray, grads: np.ndarray, fmts, scale_list, inv_list) -> np.ndarray:

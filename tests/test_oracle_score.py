@@ -234,3 +234,43 @@ def test_group_costs_and_budget_hand_examples(orc):
         assert orc.group_costs([l], np.array([[0, 1]], np.uint8), d_layer).tolist() == [0.0, d_layer[l, 1]]
     assert orc.budget_from_tau(0.1, [1.0, 2.0, 3.0]) == pytest.approx(0.01 * 14.0 / 3.0, rel=1e-15)
     assert orc.budget_from_tau(0.0, [1.0, 2.0]) == 0.0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("f", [1, 2])
+def test_fake_quant_pins(orc, dtype, f):
+    """The quantised operand z^: equals the rational nearest-grid value times the
+    scale (rounded once to fp32, then to the storage type by torch's own cast),
+    reproduces tensors already on the grid, is idempotent, and its error squares
+    to the oracle's own D."""
+    rng = np.random.default_rng(21)
+    grid = _grid(f)
+    x = (rng.standard_normal(300) * np.exp(rng.uniform(-6, 3, 300))).astype(np.float32)
+    t = torch.from_numpy(x).to(dtype)
+    v = _as_oracle_array(t)
+    a = orc.amax(v)
+    sc, iv = orc.scales(f, a)
+    zh = orc.fake_quant(v, f, sc, iv)
+    z64 = t.to(torch.float64).numpy()
+    for k in range(300):   # rational arithmetic, independent of the C code
+        y = np.float32(Fraction(float(z64[k])) * Fraction(float(iv)))
+        want = np.float32(_quantise_exact(y, grid) * Fraction(float(sc)))
+        want = torch.tensor([want]).to(dtype)
+        assert _as_oracle_array(want)[0] == zh[k], k
+    # error of z^ squares to D (fp32 storage: only the one rounding of the product differs)
+    if dtype == torch.float32:
+        g = rng.standard_normal(300).astype(np.float32)
+        seg = orc.score_segment(v, g, [f], [sc], [iv])
+        d = float(np.sum((g.astype(np.float64) * (zh.astype(np.float64) - z64)) ** 2))
+        assert d == pytest.approx(seg[1], rel=1e-5)
+    # idempotent under the same scale
+    assert np.array_equal(orc.fake_quant(zh, f, sc, iv), zh)
+    # a tensor on the grid (scale a power of two) comes back unchanged
+    gv = np.array([float(q) for _, q in grid])
+    on = (rng.choice(gv, 512) * rng.choice([-1.0, 1.0], 512) * 0.25).astype(np.float32)
+    on[0] = gv[-1] * 0.25
+    ton = torch.from_numpy(on).to(dtype)
+    von = _as_oracle_array(ton)   # every FP8 value fits the 8 significant bits of bf16
+    s2, i2 = orc.scales(f, orc.amax(von))
+    assert s2 == np.float32(0.25)
+    assert np.array_equal(orc.fake_quant(von, f, s2, i2), von)
