@@ -126,6 +126,45 @@ int ampq_set_amax(ampq_ctx *ctx, int layer_id, int operand, float amax);
  * getters return AMPQ_ERR_TIMEOUT for that score and the context stays usable. */
 int ampq_score(ampq_ctx *ctx);
 
+/* Streaming form of the same step, for calibration loops that see one sample
+ * at a time (Algorithm 1 step 2: forward and backward per calibration sample)
+ * and never hold all R per-sample weight gradients at once.
+ *   ampq_stream_begin   clears the per-sample sums of every registered layer.
+ *   ampq_stream_sample  scores ONE sample r of one operand, asynchronously on
+ *                       the stream: values/grads are device pointers to numel
+ *                       elements each (activations: sample r's slice; weights:
+ *                       the whole weight and the gradient of sample r's loss
+ *                       with respect to it), borrowed until the work has
+ *                       finished.  The operand's preset amax (ampq_set_amax) is
+ *                       used when there is one -- the static-scale case, and
+ *                       the way to score activations with one scale for all
+ *                       samples; without a preset the amax of the tensor passed
+ *                       in THIS call is measured and used.  A sample streamed
+ *                       twice is overwritten, not added.  Operands need not be
+ *                       bound.
+ *   ampq_stream_end     forms the per-layer values from whatever was streamed
+ *                       (samples never streamed count as 0); afterwards
+ *                       ampq_get_layer / ampq_get_operand / ampq_group_costs /
+ *                       ampq_select work as after ampq_score.  The amax a
+ *                       getter reports is the largest any sample used, the
+ *                       scales are those of the last sample streamed.
+ * Sums equal those of ampq_score over the same data and amax up to the order
+ * of the fp64 additions. */
+int ampq_stream_begin(ampq_ctx *ctx);
+int ampq_stream_sample(ampq_ctx *ctx, int layer_id, int operand, int r, int dtype, const void *values,
+                       const void *grads, long long numel);
+int ampq_stream_end(ampq_ctx *ctx);
+
+/* The quantised operand itself (z^ = z + z~ of Sec. 2.2): writes
+ * dec(Q(z*inv))*scale, one fp32 product stored in the operand's own dtype
+ * (bf16: round to nearest even), for numel elements; values and dev_out are
+ * device pointers (dev_out may equal values).  amax >= 0: use it; < 0: measure
+ * it over `values`.  fmt must be in the context's format list.  Asynchronous
+ * on the stream.  Used to run a model "in format f" when checking predicted
+ * against measured loss MSE (Sec. 3.2). */
+int ampq_fake_quant(ampq_ctx *ctx, int dtype, int fmt, const void *values, long long numel, float amax,
+                    void *dev_out);
+
 /* Number of kernel launches issued by the last ampq_score (diagnostics). */
 int ampq_last_launch_count(const ampq_ctx *ctx);
 

@@ -34,7 +34,7 @@ EXPORTS = [
     "ampq_last_launch_count", "ampq_set_timing", "ampq_get_timing", "ampq_get_layer", "ampq_get_operand", "ampq_export_codes",
     "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
-    "ampq_group_costs_table",
+    "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -79,6 +79,10 @@ def lib():
     L.ampq_define_group.argtypes = [vp, vp, i, vp, vp, i, ip]
     L.ampq_clear_groups.argtypes = [vp]
     L.ampq_group_costs.argtypes = [vp, i, i, vp]
+    L.ampq_stream_begin.argtypes = [vp]
+    L.ampq_stream_sample.argtypes = [vp, i, i, i, i, vp, vp, ll]
+    L.ampq_stream_end.argtypes = [vp]
+    L.ampq_fake_quant.argtypes = [vp, i, i, vp, ll, C.c_float, vp]
     L.ampq_group_costs_table.argtypes = [vp, i, vp, i, vp, i, i, vp]
     L.ampq_budget_from_tau.argtypes = [C.c_double, vp, i, dp]
     L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
@@ -204,6 +208,21 @@ class Context:
 
     def score(self):
         self._check(lib().ampq_score(self._h))
+
+    def stream_begin(self):
+        self._check(lib().ampq_stream_begin(self._h))
+
+    def stream_sample(self, layer_id: int, operand: int, r: int, dtype: int, values_ptr: int, grads_ptr: int,
+                      numel: int):
+        self._check(lib().ampq_stream_sample(self._h, layer_id, operand, r, dtype, C.c_void_p(values_ptr),
+                                             C.c_void_p(grads_ptr), numel))
+
+    def stream_end(self):
+        self._check(lib().ampq_stream_end(self._h))
+
+    def fake_quant(self, dtype: int, fmt: int, values_ptr: int, numel: int, amax: float, out_ptr: int):
+        self._check(lib().ampq_fake_quant(self._h, dtype, fmt, C.c_void_p(values_ptr), numel, amax,
+                                          C.c_void_p(out_ptr)))
 
     def last_launch_count(self) -> int:
         return lib().ampq_last_launch_count(self._h)

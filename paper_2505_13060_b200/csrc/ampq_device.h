@@ -73,6 +73,18 @@ struct Layer {
 // Layer output block layout (doubles): s_r[R], s_mean, d_meas_r[R*F], d_model[F], d_meas[F]
 inline int layer_block_doubles(int R, int F) { return R + 1 + R * F + 2 * F; }
 
+// The tables of a one-tensor, one-sample scoring job (streaming calibration,
+// fake quantisation): what a full score keeps in separate arrays, for one segment.
+struct SegmentJob {
+    Tensor tensor;
+    long long tile_begin[2];       // scoring tiles {0, ntiles}
+    long long amax_tile_begin[2];  // amax tiles {0, n_amax_tiles}
+    Segment segment;
+    unsigned amax_bits;
+    int flag;                      // 1: the tensor held Inf/NaN
+    float scales[2 * kMaxLow];
+};
+
 struct LaunchStatus {
     int nonfinite;  // set when some tensor's amax is Inf/NaN
     int timeout;    // set when a wait inside the scoring kernel ran out

@@ -788,6 +788,78 @@ __global__ void codes_kernel(const void* __restrict__ values, long long n, const
 }
 
 // ---------------------------------------------------------------------------
+// one-segment jobs (streaming calibration, fake quantisation)
+
+__global__ void job_prepare_kernel(SegmentJob* job, const void* values, const void* grads, long long n, int dtype,
+                                   float amax_preset, long long ntiles, long long namax) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    Tensor t;
+    t.values = values;
+    t.grads = grads;
+    t.numel = n;
+    t.seg_len = n;
+    t.grad_stride = n;
+    t.partial_base = 0;
+    t.tiles_per_seg = (int)ntiles;
+    t.R = 1;
+    t.per_sample = 1;
+    t.dtype = dtype;
+    t.rgroups = 1;
+    t.seg_base = 0;
+    t.amax_preset = amax_preset;
+    t.pad = 0;
+    job->tensor = t;
+    job->tile_begin[0] = 0;
+    job->tile_begin[1] = ntiles;
+    job->amax_tile_begin[0] = 0;
+    job->amax_tile_begin[1] = namax;
+    job->segment.first_slot = 0;
+    job->segment.count = (int)ntiles;
+    job->segment.pad = 0;
+    job->amax_bits = amax_preset >= 0.0f ? __float_as_uint(amax_preset) : 0u;
+    job->flag = 0;
+}
+
+// Folds a finished job into the per-tensor arrays of the context: the largest
+// amax any sample used, a sticky non-finite flag, the scales of the last sample.
+__global__ void job_fold_kernel(const SegmentJob* job, int tensor, unsigned* amax_bits, int* flags, float* scales) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    atomicMax(amax_bits + tensor, job->amax_bits);
+    if (job->flag) flags[tensor] = 1;
+    for (int k = 0; k < 2 * kMaxLow; ++k) scales[tensor * 2 * kMaxLow + k] = job->scales[k];
+}
+
+// The quantised operand itself: out_k = dec(Q(z_k * inv)) * scale as one fp32
+// product, stored in the operand's own type (bf16: round to nearest even).
+template <int DT, int FMT>
+__global__ void fake_quant_kernel(const void* __restrict__ values, long long n, const float* __restrict__ scale_pair,
+                                  void* __restrict__ out) {
+    const float scale = scale_pair[0], inv = scale_pair[1];
+    const long long npairs = (n + 1) / 2;
+    for (long long p = blockIdx.x * (long long)blockDim.x + threadIdx.x; p < npairs;
+         p += (long long)gridDim.x * blockDim.x) {
+        const long long i = 2 * p;
+        const bool two = i + 1 < n;
+        float2 z = make_float2(Elem<DT>::load(values, i), two ? Elem<DT>::load(values, i + 1) : 0.0f);
+        float2 y = __fmul2_rn(z, make_float2(inv, inv));
+        float2 dq = decode_pair<FMT>(cast_pair<FMT>(y.x, y.y));
+        float2 zh = __fmul2_rn(dq, make_float2(scale, scale));
+        if (DT == 0) {
+            float* o = reinterpret_cast<float*>(out);
+            o[i] = zh.x;
+            if (two) o[i + 1] = zh.y;
+        } else {
+            unsigned short* o = reinterpret_cast<unsigned short*>(out);
+            unsigned short lo, hi;
+            asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(lo) : "f"(zh.x));
+            asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(hi) : "f"(zh.y));
+            o[i] = lo;
+            if (two) o[i + 1] = hi;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // host launchers
 
 cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, LaunchStatus* status,
@@ -879,6 +951,31 @@ cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParam
                            double* layer_out, cudaStream_t st) {
     if (L <= 0) return cudaSuccess;
     combine_kernel<<<(L + 127) / 128, 128, 0, st>>>(layers, L, F, prm, seg_out, layer_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_job_prepare(SegmentJob* job, const void* values, const void* grads, long long n, int dtype,
+                               float amax_preset, long long ntiles, long long namax, cudaStream_t st) {
+    job_prepare_kernel<<<1, 32, 0, st>>>(job, values, grads, n, dtype, amax_preset, ntiles, namax);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_job_fold(const SegmentJob* job, int tensor, unsigned* amax_bits, int* flags, float* scales,
+                            cudaStream_t st) {
+    job_fold_kernel<<<1, 32, 0, st>>>(job, tensor, amax_bits, flags, scales);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fake_quant(int dtype, int fmt_mask, const void* values, long long n, const float* scale_pair,
+                              void* out, cudaStream_t st) {
+    if (n <= 0) return cudaSuccess;
+    long long blocks = ((n + 1) / 2 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    const unsigned grid = (unsigned)blocks;
+    if (dtype == 0 && fmt_mask == kMaskE4M3) fake_quant_kernel<0, kMaskE4M3><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else if (dtype == 0) fake_quant_kernel<0, kMaskE5M2><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else if (fmt_mask == kMaskE4M3) fake_quant_kernel<1, kMaskE4M3><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
+    else fake_quant_kernel<1, kMaskE5M2><<<grid, 256, 0, st>>>(values, n, scale_pair, out);
     return cudaGetLastError();
 }
 

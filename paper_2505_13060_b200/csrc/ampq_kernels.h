@@ -34,6 +34,15 @@ cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const doubl
                             cudaStream_t st);
 cudaError_t launch_combine(const Layer* layers, int L, int F, const CombineParams& prm, const double* seg_out,
                            double* layer_out, cudaStream_t st);
+// One-segment jobs: fill a job's tables on the device, fold its amax / flag /
+// scales into per-tensor arrays afterwards.
+cudaError_t launch_job_prepare(SegmentJob* job, const void* values, const void* grads, long long n, int dtype,
+                               float amax_preset, long long ntiles, long long namax, cudaStream_t st);
+cudaError_t launch_job_fold(const SegmentJob* job, int tensor, unsigned* amax_bits, int* flags, float* scales,
+                            cudaStream_t st);
+// scale_pair = {scale, inv_scale} on the device; out has the operand's dtype.
+cudaError_t launch_fake_quant(int dtype, int fmt_mask, const void* values, long long n, const float* scale_pair,
+                              void* out, cudaStream_t st);
 cudaError_t launch_codes(int dtype, int fmt_mask, const void* values, long long n, const float* scale_pair,
                          unsigned char* out, cudaStream_t st);
 

@@ -136,6 +136,13 @@ struct ampq_ctx {
     PinBuf<double> h_seg_out, h_layer_out;
     PinBuf<LaunchStatus> h_status;
 
+    // streaming calibration (ampq_stream_*) and fake quantisation
+    bool streaming = false;
+    std::vector<int> stream_seg_base;   // [2*layer + operand] -> first segment (sample 0)
+    DevBuf<SegmentJob> d_jobs;          // one job per (tensor, sample) of a streaming pass
+    DevBuf<double> d_job_partials;      // per-tile partials of the job in flight (jobs are ordered on the stream)
+    DevBuf<SegmentJob> d_fq_job;        // tables of a fake-quantisation call
+
     bool timing = false;            // record CUDA events around the kernels of a score
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     bool ev_valid = false;
@@ -392,6 +399,39 @@ int group_costs_impl(ampq_ctx* ctx, const Group& g, int d_mode, double* d_out) {
     return AMPQ_OK;
 }
 
+// Per-layer combine and the asynchronous read-back of every small result.
+int combine_and_read_back(ampq_ctx* ctx, int T, int L, int S) {
+    const int nacc = ctx->F;
+    cudaStream_t st = ctx->stream;
+    CombineParams prm{};
+    prm.nacc = nacc;
+    for (int f = 1; f < ctx->F; ++f) {
+        prm.alpha[f] = std::ldexp(1.0, -2 * mantissa_bits_of(ctx->fmt[f])) / 12.0;
+        prm.acc_of_fmt[f] = 1 + ctx->slot_of_fmt[f];
+    }
+    AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, prm, ctx->d_seg_out.p, ctx->d_layer_out.p, st), "combine");
+    ++ctx->launches;
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_scales.p, ctx->d_scales.p, (size_t)T * 2 * kMaxLow * sizeof(float), cudaMemcpyDeviceToHost, st), "D2H scales");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_flags.p, ctx->d_flags.p, T * sizeof(int), cudaMemcpyDeviceToHost, st), "D2H flags");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_seg_out.p, ctx->d_seg_out.p, (size_t)S * nacc * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H segments");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_layer_out.p, ctx->d_layer_out.p, (size_t)ctx->layer_out_doubles * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H layers");
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_status.p, ctx->d_status.p, sizeof(LaunchStatus), cudaMemcpyDeviceToHost, st), "D2H status");
+    return AMPQ_OK;
+}
+
+// Runs one (tensor, sample) job through amax / scales on the stream; the
+// caller launches what follows.  job is a device pointer.
+int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, int dtype, const void* values, const void* grads,
+                        long long numel, float preset, long long ntiles) {
+    cudaStream_t st = ctx->stream;
+    const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
+    AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, st), "job_prepare");
+    AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st), "amax");
+    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, ctx->d_status.p, st), "scales");
+    return AMPQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -450,6 +490,7 @@ int ampq_destroy(ampq_ctx* ctx) {
         ctx->d_segs.release(); ctx->d_lay.release(); ctx->d_amax_bits.release(); ctx->d_scales.release();
         ctx->d_partials.release(); ctx->d_flags.release(); ctx->d_seg_out.release();
         ctx->d_layer_out.release(); ctx->d_status.release();
+        ctx->d_jobs.release(); ctx->d_job_partials.release(); ctx->d_fq_job.release();
         ctx->h_amax_bits.release(); ctx->h_scales.release(); ctx->h_flags.release();
         ctx->h_seg_out.release(); ctx->h_layer_out.release(); ctx->h_status.release();
         for (int i = 0; i < 6; ++i)
@@ -535,6 +576,7 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
         ctx->pending = false;
     }
+    ctx->streaming = false;  // a full score ends any streaming pass
     if (ctx->dirty) {
         ctx->scored = false;
         if ((rc = build_tables(ctx))) return rc;
@@ -569,20 +611,7 @@ int ampq_score(ampq_ctx* ctx) {
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");
         AMPQ_CUDA(launch_finalize(ctx->d_segs.p, S, nacc, ctx->d_partials.p, ctx->d_seg_out.p, st), "finalize");
         ++ctx->launches;
-        CombineParams prm{};
-        prm.nacc = nacc;
-        for (int f = 1; f < ctx->F; ++f) {
-            prm.alpha[f] = std::ldexp(1.0, -2 * mantissa_bits_of(ctx->fmt[f])) / 12.0;
-            prm.acc_of_fmt[f] = 1 + ctx->slot_of_fmt[f];
-        }
-        AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, prm, ctx->d_seg_out.p, ctx->d_layer_out.p, st), "combine");
-        ++ctx->launches;
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_scales.p, ctx->d_scales.p, (size_t)T * 2 * kMaxLow * sizeof(float), cudaMemcpyDeviceToHost, st), "D2H scales");
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_flags.p, ctx->d_flags.p, T * sizeof(int), cudaMemcpyDeviceToHost, st), "D2H flags");
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_seg_out.p, ctx->d_seg_out.p, (size_t)S * nacc * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H segments");
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_layer_out.p, ctx->d_layer_out.p, (size_t)ctx->layer_out_doubles * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H layers");
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_status.p, ctx->d_status.p, sizeof(LaunchStatus), cudaMemcpyDeviceToHost, st), "D2H status");
+        if ((rc = combine_and_read_back(ctx, T, L, S))) return rc;
         if (tm) {
             AMPQ_CUDA(cudaEventRecord(ctx->ev[5], st), "cudaEventRecord");
             ctx->ev_valid = true;
@@ -590,6 +619,148 @@ int ampq_score(ampq_ctx* ctx) {
     }
     ctx->scored = true;
     ctx->pending = T > 0;
+    return AMPQ_OK;
+}
+
+int ampq_stream_begin(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    if (ctx->pending) {
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        ctx->pending = false;
+    }
+    // tables over EVERY registered layer: tensor 2*l + operand, one segment per sample
+    ctx->tens.clear(); ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
+    ctx->stream_seg_base.clear();
+    int out_off = 0, nseg = 0;
+    for (size_t li = 0; li < ctx->layers.size(); ++li) {
+        LayerRec& l = ctx->layers[li];
+        Layer ly{};
+        ly.R = l.R;
+        ly.out_off = out_off;
+        out_off += layer_block_doubles(l.R, ctx->F);
+        for (int k = 0; k < 2; ++k) {
+            Tensor t{};
+            t.R = l.R;
+            t.seg_base = nseg;
+            t.amax_preset = l.op[k].amax_preset;
+            l.op[k].tensor = (int)ctx->tens.size();
+            ctx->stream_seg_base.push_back(nseg);
+            if (k == 0) { ly.seg_base0 = nseg; ly.tensor0 = l.op[k].tensor; }
+            else { ly.seg_base1 = nseg; ly.tensor1 = l.op[k].tensor; }
+            ctx->tens.push_back(t);
+            nseg += l.R;
+        }
+        l.scored = (int)ctx->lay.size();
+        ctx->lay.push_back(ly);
+        ctx->scored_layer_ids.push_back((int)li);
+    }
+    ctx->layer_out_doubles = out_off;
+    const size_t T = ctx->tens.size(), L = ctx->lay.size(), S = (size_t)nseg;
+    const int nacc = ctx->F;
+    AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
+    AMPQ_CUDA(ctx->d_amax_bits.ensure(T), "cudaMalloc(amax)");
+    AMPQ_CUDA(ctx->d_scales.ensure(T * 2 * kMaxLow), "cudaMalloc(scales)");
+    AMPQ_CUDA(ctx->d_flags.ensure(T), "cudaMalloc(flags)");
+    AMPQ_CUDA(ctx->d_seg_out.ensure(S * nacc), "cudaMalloc(seg_out)");
+    AMPQ_CUDA(ctx->d_layer_out.ensure((size_t)out_off), "cudaMalloc(layer_out)");
+    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
+    AMPQ_CUDA(ctx->d_jobs.ensure(S), "cudaMalloc(jobs)");
+    AMPQ_CUDA(ctx->h_amax_bits.ensure(T), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_scales.ensure(T * 2 * kMaxLow), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_flags.ensure(T), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_seg_out.ensure(S * nacc), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_layer_out.ensure((size_t)out_off), "cudaMallocHost");
+    AMPQ_CUDA(ctx->h_status.ensure(1), "cudaMallocHost");
+    cudaStream_t st = ctx->stream;
+    if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
+    if (T) {
+        AMPQ_CUDA(cudaMemsetAsync(ctx->d_amax_bits.p, 0, T * sizeof(unsigned), st), "memset amax");
+        AMPQ_CUDA(cudaMemsetAsync(ctx->d_flags.p, 0, T * sizeof(int), st), "memset flags");
+        AMPQ_CUDA(cudaMemsetAsync(ctx->d_scales.p, 0, T * 2 * kMaxLow * sizeof(float), st), "memset scales");
+    }
+    if (S) AMPQ_CUDA(cudaMemsetAsync(ctx->d_seg_out.p, 0, S * nacc * sizeof(double), st), "memset seg_out");
+    AMPQ_CUDA(cudaMemsetAsync(ctx->d_status.p, 0, sizeof(LaunchStatus), st), "memset status");
+    ctx->streaming = true;
+    ctx->scored = false;
+    ctx->dirty = true;  // a later ampq_score rebuilds its own tables
+    ctx->launches = 0;
+    ctx->ev_valid = false;
+    return AMPQ_OK;
+}
+
+int ampq_stream_sample(ampq_ctx* ctx, int layer_id, int operand, int r, int dtype, const void* values,
+                       const void* grads, long long numel) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (!ctx->streaming) return fail(ctx, AMPQ_ERR_STATE, "ampq_stream_sample outside ampq_stream_begin / ampq_stream_end");
+    if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
+    if (dtype != AMPQ_F32 && dtype != AMPQ_BF16) return fail(ctx, AMPQ_ERR_INVALID, "unknown dtype");
+    const LayerRec& l = ctx->layers[layer_id];
+    if (l.scored < 0 || 2 * (size_t)layer_id + 1 >= ctx->stream_seg_base.size())
+        return fail(ctx, AMPQ_ERR_STATE, "layer was registered after ampq_stream_begin");
+    if (r < 0 || r >= l.R) return fail(ctx, AMPQ_ERR_INVALID, "sample index outside [0, R)");
+    if (numel < 0 || (numel > 0 && (!values || !grads))) return fail(ctx, AMPQ_ERR_INVALID, "bad tensor");
+    const int es = dtype == AMPQ_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(values) % es) || (reinterpret_cast<uintptr_t>(grads) % es))
+        return fail(ctx, AMPQ_ERR_ALIGN, "tensor pointer not aligned to its element size");
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    const int nacc = ctx->F;
+    const int tensor = 2 * layer_id + operand;
+    const int seg = ctx->stream_seg_base[tensor] + r;
+    const int shift = pick_tile_shift(numel, ctx->max_ctas);
+    const long long ntiles = (numel + (1LL << shift) - 1) >> shift;
+    if (ntiles > 0x7FFFFFFFLL) return fail(ctx, AMPQ_ERR_TOO_LARGE, "more than 2^31-1 tiles in one sample");
+    AMPQ_CUDA(ctx->d_job_partials.ensure((size_t)ntiles * nacc + 1), "cudaMalloc(job partials)");
+    SegmentJob* job = ctx->d_jobs.p + seg;
+    cudaStream_t st = ctx->stream;
+    if ((rc = job_amax_and_scales(ctx, job, dtype, values, grads, numel, l.op[operand].amax_preset, ntiles))) return rc;
+    AMPQ_CUDA(launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &job->tensor, job->tile_begin, 1, ntiles, shift, ctx->max_ctas,
+                           ctx->fmask, job->scales, ctx->d_job_partials.p, ctx->d_status.p, st), "score");
+    AMPQ_CUDA(launch_finalize(&job->segment, 1, nacc, ctx->d_job_partials.p, ctx->d_seg_out.p + (size_t)seg * nacc, st), "finalize");
+    AMPQ_CUDA(launch_job_fold(job, tensor, ctx->d_amax_bits.p, ctx->d_flags.p, ctx->d_scales.p, st), "job_fold");
+    ctx->launches += numel > 0 ? 6 : 4;
+    return AMPQ_OK;
+}
+
+int ampq_stream_end(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    if (!ctx->streaming) return fail(ctx, AMPQ_ERR_STATE, "ampq_stream_end without ampq_stream_begin");
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    int nseg = 0;
+    for (const auto& ly : ctx->lay) nseg += 2 * ly.R;
+    const int T = (int)ctx->tens.size(), L = (int)ctx->lay.size();
+    int rc = AMPQ_OK;
+    if (T > 0 && (rc = combine_and_read_back(ctx, T, L, nseg))) return rc;
+    ctx->streaming = false;
+    ctx->scored = true;
+    ctx->pending = T > 0;
+    return AMPQ_OK;
+}
+
+int ampq_fake_quant(ampq_ctx* ctx, int dtype, int fmt, const void* values, long long numel, float amax, void* dev_out) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    if (dtype != AMPQ_F32 && dtype != AMPQ_BF16) return fail(ctx, AMPQ_ERR_INVALID, "unknown dtype");
+    if (numel < 0 || (numel > 0 && (!values || !dev_out))) return fail(ctx, AMPQ_ERR_INVALID, "bad tensor");
+    if (amax != amax || std::isinf(amax)) return fail(ctx, AMPQ_ERR_INVALID, "amax must be finite");
+    int f = -1;
+    for (int k = 1; k < ctx->F; ++k)
+        if (ctx->fmt[k] == fmt) f = k;
+    if (f < 0) return fail(ctx, AMPQ_ERR_INVALID, "format is not in the context's format list");
+    const int es = dtype == AMPQ_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(values) % es) || (reinterpret_cast<uintptr_t>(dev_out) % es))
+        return fail(ctx, AMPQ_ERR_ALIGN, "tensor pointer not aligned to its element size");
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    AMPQ_CUDA(ctx->d_fq_job.ensure(1), "cudaMalloc(job)");
+    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
+    int rc = job_amax_and_scales(ctx, ctx->d_fq_job.p, dtype, values, values, numel, amax >= 0.0f ? amax : -1.0f, 0);
+    if (rc) return rc;
+    const float* pair = ctx->d_fq_job.p->scales + ctx->slot_of_fmt[f] * 2;
+    AMPQ_CUDA(launch_fake_quant(dtype, fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2, values, numel, pair, dev_out, ctx->stream), "fake_quant");
     return AMPQ_OK;
 }
 

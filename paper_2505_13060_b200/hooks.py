@@ -1,0 +1,123 @@
+"""Calibration of a PyTorch model through module hooks (Algorithm 1 step 2:
+"wrap the model", then one high-precision forward and backward per sample).
+
+``Calibrator`` registers every ``torch.nn.Linear`` of a model as a layer of a
+scoring context.  While a sample runs, a forward hook keeps the layer input X
+and a backward hook receives dL/dX and dL/dY; the sample's weight gradient
+dL/dW = dL/dY^T X is formed by a torch matmul (the GEMM that produces a gradient
+is not part of the scoring path) and both operands of the layer are streamed to
+``ampq_stream_sample``, so the R per-sample weight gradients never exist at the
+same time.  Everything the method computes happens in the CUDA library; this
+module only moves pointers.
+
+``quantised(...)`` runs the model with chosen layers' inputs and weights replaced
+by their FP8-rounded values (``ampq_fake_quant``), which is how the predicted
+loss MSE is checked against a measured one (Sec. 3.2).
+"""
+from __future__ import annotations
+
+import contextlib
+
+import torch
+
+from . import binding as ampq
+
+
+class Calibrator:
+    def __init__(self, ctx: "ampq.Context", model: torch.nn.Module, R: int):
+        self.ctx, self.model, self.R = ctx, model, R
+        self.modules, self.layer_ids = [], []
+        for name, m in model.named_modules():
+            if isinstance(m, torch.nn.Linear):
+                self.modules.append((name, m))
+                self.layer_ids.append(ctx.register_layer(ampq.LINEAR, name, R))
+        self._r = None
+        self._x = {}
+        self._keep = []   # tensors borrowed by the library until the stream has caught up
+        self._handles = []
+
+    # -- hooks ----------------------------------------------------------------
+    def _fwd(self, idx):
+        def hook(module, inputs, output):
+            if self._r is not None:
+                self._x[idx] = inputs[0].detach()
+        return hook
+
+    def _bwd(self, idx):
+        def hook(module, grad_input, grad_output):
+            if self._r is None:
+                return
+            x = self._x.pop(idx).contiguous()
+            gy = grad_output[0].detach()
+            gx = grad_input[0]
+            w = module.weight.detach().contiguous()
+            if gx is None:   # the model input needs no gradient: form dL/dX here
+                gx = gy.reshape(-1, gy.shape[-1]) @ w
+            gx = gx.detach().reshape(x.shape).contiguous()
+            gw = (gy.reshape(-1, gy.shape[-1]).t() @ x.reshape(-1, x.shape[-1])).contiguous()
+            code = ampq.torch_dtype_code(x)
+            lid = self.layer_ids[idx]
+            self.ctx.stream_sample(lid, 0, self._r, code, x.data_ptr(), gx.data_ptr(), x.numel())
+            self.ctx.stream_sample(lid, 1, self._r, code, w.data_ptr(), gw.data_ptr(), w.numel())
+            self._keep += [x, gx, w, gw]
+        return hook
+
+    def begin(self):
+        self._handles = []
+        for idx, (_, m) in enumerate(self.modules):
+            self._handles.append(m.register_forward_hook(self._fwd(idx)))
+            self._handles.append(m.register_full_backward_hook(self._bwd(idx)))
+        self.ctx.stream_begin()
+
+    @contextlib.contextmanager
+    def sample(self, r: int):
+        """Run one sample's forward and backward inside this block."""
+        self._r = r
+        try:
+            yield
+        finally:
+            self._r = None
+            self._x.clear()
+
+    def end(self):
+        self.ctx.stream_end()
+        res = [self.ctx.get_layer(lid) for lid in self.layer_ids]   # synchronises: the borrowed tensors are free
+        self._keep.clear()
+        for h in self._handles:
+            h.remove()
+        self._handles = []
+        return res
+
+    # -- running the model in a low-precision configuration --------------------
+    @contextlib.contextmanager
+    def quantised(self, fmt_of_layer, amax_x=None):
+        """Inside this block layer i (index into ``modules``) runs with its input and
+        weight rounded to format ``fmt_of_layer[i]`` (0 leaves it alone).
+        ``amax_x[i]`` is the static amax of the layer's input (measured per call if
+        absent); the weight's amax is always measured."""
+        saved, handles = [], []
+        for idx, (_, m) in enumerate(self.modules):
+            fmt = fmt_of_layer[idx]
+            if not fmt:
+                continue
+            w = m.weight.data
+            saved.append((m, w.clone()))
+            self.ctx.fake_quant(ampq.torch_dtype_code(w), fmt, w.data_ptr(), w.numel(), -1.0, w.data_ptr())
+
+            def pre(module, inputs, fmt=fmt, a=(-1.0 if amax_x is None else float(amax_x[idx]))):
+                x = inputs[0].contiguous()
+                out = torch.empty_like(x)
+                self.ctx.fake_quant(ampq.torch_dtype_code(x), fmt, x.data_ptr(), x.numel(), a, out.data_ptr())
+                self._keep.append(x)
+                return (out,) + tuple(inputs[1:])
+
+            handles.append(m.register_forward_pre_hook(pre))
+        try:
+            yield
+        finally:
+            torch.cuda.current_stream().synchronize()
+            for h in handles:
+                h.remove()
+            for m, w in saved:
+                m.weight.data.copy_(w)
+            self._keep.clear()

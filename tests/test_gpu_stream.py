@@ -1,0 +1,185 @@
+"""GPU parity of the streaming calibration calls, the fake quantisation, and a
+miniature of the paper's model validation (Sec. 3.2): predicted against
+measured loss MSE on a random toy MLP calibrated through module hooks."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close, compare_layer, oracle_layer
+from paper_2505_13060_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+E4M3, E5M2 = 1, 2
+
+
+def _ctx(ampq, fmts):
+    ctx = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
+    ctx.set_formats(list(fmts))
+    return ctx
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_streamed_samples_match_oracle_and_full_score(ampq, orc, dtype):
+    """Sample by sample with a static amax on the activations and a measured one
+    on the weights: every value equals the oracle's, and the full score of the
+    same tensors gives the same numbers up to the order of fp64 additions."""
+    R = 3
+    specs = [synth.LayerSpec("s%d" % i, synth.LINEAR, R, dtype,
+                             synth.OperandSpec((R, nx), True, 1.0, 1e-3, "normal", ("element", 0.01, 20.0)),
+                             synth.OperandSpec((nw,), False, 0.02, 1e-3))
+             for i, (nx, nw) in enumerate([(70001, 40000), (3 * 32768, 65536 + 7), (5, 1 << 20)])]
+    lts = [synth.make_layer(s, "cuda", seed=12, layer=i) for i, s in enumerate(specs)]
+    code = ampq.torch_dtype_code(lts[0].values[0])
+    ctx = _ctx(ampq, (0, E4M3, E5M2))
+    ids = [ctx.register_layer(lt.spec.kind, lt.spec.name, R) for lt in lts]
+    amax_x = [float(lt.values[0].float().abs().max()) for lt in lts]   # plumbing: a static scale from anywhere
+    for lid, a in zip(ids, amax_x):
+        ctx.set_amax(lid, 0, a)
+    ctx.stream_begin()
+    for r in range(R):   # samples arrive one at a time, layers in any order
+        for lid, lt in reversed(list(zip(ids, lts))):
+            x, gx = lt.values[0][r], lt.grads[0][r]
+            ctx.stream_sample(lid, 0, r, code, x.data_ptr(), gx.data_ptr(), x.numel())
+            w, gw = lt.values[1], lt.grads[1][r]
+            ctx.stream_sample(lid, 1, r, code, w.data_ptr(), gw.data_ptr(), w.numel())
+    ctx.stream_end()
+    streamed = []
+    for lid, lt, a in zip(ids, lts, amax_x):
+        ref = oracle_layer(orc, lt, [E4M3, E5M2], amax_presets=(a, None))
+        streamed.append((compare_layer(ampq, ctx, lid, ref, 3, "streamed " + lt.spec.name),
+                         ctx.get_operand(lid, 0), ctx.get_operand(lid, 1)))
+    # a sample streamed twice is overwritten, not added; an unstreamed one counts as 0
+    ctx.stream_begin()
+    lt = lts[0]
+    for _ in range(2):
+        ctx.stream_sample(ids[0], 0, 1, code, lt.values[0][1].data_ptr(), lt.grads[0][1].data_ptr(), lt.values[0][1].numel())
+    ctx.stream_end()
+    o = ctx.get_operand(ids[0], 0)
+    assert o[1].tobytes() == streamed[0][1][1].tobytes() and not o[0].any() and not o[2].any()
+    assert not ctx.get_operand(ids[1], 0).any()
+    # the full score over the same tensors
+    for lid, lt in zip(ids, lts):
+        ampq.bind_layer_tensors(ctx, lid, lt)
+    ctx.score()
+    for lid, (got, o0, o1) in zip(ids, streamed):
+        full = ctx.get_layer(lid)
+        assert full["amax"].tobytes() == got["amax"].tobytes()
+        assert_close(full["s_per_sample"], got["s_per_sample"], "full vs streamed s", tol=1e-12)
+        assert_close(full["d_meas_per_sample"], got["d_meas_per_sample"], "full vs streamed d", tol=1e-12)
+    # calls out of order are refused
+    L = ampq.lib()
+    assert L.ampq_stream_sample(ctx._h, ids[0], 0, 0, code, lt.values[0].data_ptr(), lt.grads[0].data_ptr(), 8) == ampq.ERR_STATE
+    assert L.ampq_stream_end(ctx._h) == ampq.ERR_STATE
+    ctx.stream_begin()
+    assert L.ampq_stream_sample(ctx._h, ids[0], 0, R, code, lt.values[0].data_ptr(), lt.grads[0].data_ptr(), 8) == ampq.ERR_INVALID
+    assert L.ampq_stream_sample(ctx._h, ids[0], 2, 0, code, lt.values[0].data_ptr(), lt.grads[0].data_ptr(), 8) == ampq.ERR_INVALID
+    ctx.stream_end()
+    ctx.destroy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_fake_quant_bit_exact(ampq, orc, dtype, fmt):
+    g = torch.Generator(device="cuda").manual_seed(31)
+    ctx = _ctx(ampq, (0, E4M3, E5M2))
+    code = 0 if dtype == torch.float32 else 1
+    for n, amax in ((100003, -1.0), (1, -1.0), (65536, 1.5), (0, -1.0)):
+        x = (torch.empty(max(n, 1), device="cuda").normal_(0, 1, generator=g)
+             * torch.exp(torch.empty(max(n, 1), device="cuda").uniform_(-8, 2, generator=g))).to(dtype)[:n]
+        out = torch.full((max(n, 1),), 7.0, dtype=dtype, device="cuda")[:n]
+        ctx.fake_quant(code, fmt, x.data_ptr(), n, amax, out.data_ptr())
+        torch.cuda.synchronize()
+        if n == 0:
+            continue
+        host = synth.to_numpy(x)
+        a = orc.amax(host) if amax < 0 else np.float32(amax)
+        sc, iv = orc.scales(fmt, a)
+        want = orc.fake_quant(host, fmt, sc, iv)
+        assert np.array_equal(synth.to_numpy(out).view(want.dtype), want), (n, amax)
+        # in place
+        ctx.fake_quant(code, fmt, x.data_ptr(), n, float(a), x.data_ptr())
+        torch.cuda.synchronize()
+        assert np.array_equal(synth.to_numpy(x).view(want.dtype), want)
+    with pytest.raises(ampq.AmpqError):
+        _ctx(ampq, (0, E4M3)).fake_quant(code, E5M2, out.data_ptr(), 0, -1.0, out.data_ptr())
+    ctx.destroy()
+
+
+def test_toy_mlp_hooks_and_predicted_vs_measured_loss_mse(ampq, orc):
+    """A random 4-layer MLP, R = 48 samples of 64 tokens.  Calibrate through the
+    hooks (first pass: the amax of every layer input over all samples; second
+    pass: scores with that static scale), check one layer against the oracle
+    from tensors captured independently, then run the model with every layer in
+    E4M3 and compare the measured loss MSE with the predicted one.  The first-order
+    model says E[(g^ - g)^2] = sum_l d_l; per sample the squared sum of many
+    small independent errors is chi-square distributed around it, so the mean
+    over the samples must land within a factor of two."""
+    from paper_2505_13060_b200 import hooks
+
+    torch.manual_seed(0)
+    R, tokens, width = 48, 64, 256
+    model = torch.nn.Sequential(torch.nn.Linear(width, width), torch.nn.GELU(), torch.nn.Linear(width, width),
+                                torch.nn.GELU(), torch.nn.Linear(width, width), torch.nn.GELU(),
+                                torch.nn.Linear(width, 16)).cuda()
+    xs = torch.randn(R, tokens, width, device="cuda")
+    ys = torch.randint(0, 16, (R, tokens), device="cuda")
+
+    def loss_of(r):
+        return torch.nn.functional.cross_entropy(model(xs[r]), ys[r])
+
+    ctx = _ctx(ampq, (0, E4M3))
+    cal = hooks.Calibrator(ctx, model, R)
+    assert len(cal.layer_ids) == 4
+    # pass 1: per-sample scales; the amax reported is the largest over the samples
+    cal.begin()
+    for r in range(R):
+        with cal.sample(r):
+            loss_of(r).backward()
+    first = cal.end()
+    amax_x = [float(res["amax"][0]) for res in first]
+    for lid, a in zip(cal.layer_ids, amax_x):
+        ctx.set_amax(lid, 0, a)
+    # pass 2: one static scale per layer input
+    captured = {}
+    h1 = model[2].register_forward_hook(lambda m, i, o: captured.setdefault("x", []).append(i[0].detach().clone()))
+    h2 = model[2].register_full_backward_hook(
+        lambda m, gi, go: captured.setdefault("g", []).append((gi[0].detach().clone(), go[0].detach().clone())))
+    g = []
+    cal.begin()
+    for r in range(R):
+        with cal.sample(r):
+            l = loss_of(r)
+            l.backward()
+            g.append(float(l.detach()))
+    res = cal.end()
+    h1.remove(); h2.remove()
+    # layer 1 (the second Linear) against the oracle, from independently captured tensors
+    X = torch.stack(captured["x"])
+    GX = torch.stack([a for a, _ in captured["g"]])
+    GW = torch.stack([gy.t() @ x for x, (_, gy) in zip(captured["x"], captured["g"])])
+    assert float(X.abs().max()) == amax_x[1]
+
+    class LT:
+        pass
+
+    lt = LT()
+    lt.spec = synth.LayerSpec("fc1", synth.LINEAR, R, torch.float32, synth.OperandSpec((R, tokens, width), True),
+                              synth.OperandSpec((width, width), False))
+    lt.values = [X, model[2].weight.detach()]
+    lt.grads = [GX, GW]
+    compare_layer(ampq, ctx, cal.layer_ids[1], oracle_layer(orc, lt, [E4M3], amax_presets=(amax_x[1], None)), 2, "hooked fc1")
+    # predicted: every layer in E4M3
+    d_meas = sum(r_["d_meas"][1] for r_ in res)
+    d_model = sum(r_["d_model"][1] for r_ in res)
+    # measured: run the model with inputs and weights rounded to E4M3
+    with torch.no_grad(), cal.quantised([E4M3] * 4, amax_x):
+        gq = [float(loss_of(r)) for r in range(R)]
+    measured = float(np.mean((np.array(gq) - np.array(g)) ** 2))
+    assert measured > 0
+    assert 0.5 < measured / d_meas < 2.0, (measured, d_meas, d_model)
+    assert 0.15 < measured / d_model < 1.2, (measured, d_meas, d_model)
+    # nothing is left quantised
+    with torch.no_grad():
+        assert [float(loss_of(r)) for r in range(3)] == g[:3]
+    ctx.destroy()
