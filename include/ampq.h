@@ -242,6 +242,43 @@ int ampq_select_tables(int J, const int *P, const long long *off, const double *
                        const double *d, double budget, int *p_out, double *c_total,
                        double *d_total);
 
+/* Partition of a model's computation graph into sequential sub-graphs
+ * (Appendix B, Algorithm 2).  Vertices 0..n-1, directed edges edge_src[e] ->
+ * edge_dst[e]; the graph must be acyclic with exactly one sink (the end
+ * vertex); a start vertex is put in front of every source.  Every vertex that
+ * all start -> end paths run through closes a sub-graph; a vertex belongs to
+ * the sub-graph closed by the first such vertex it reaches.  group_of[v] is the
+ * index (0, 1, ... in execution order) of the sub-graph of quantisable vertex v
+ * and -1 for the others; sub-graphs without a quantisable vertex get no index.
+ * Residual connections drawn as edges merge everything they span into one
+ * sub-graph; leave them out to split a transformer layer as the paper's figure
+ * does.  Host pointers.  AMPQ_ERR_INVALID for a cycle, several sinks or a bad
+ * edge. */
+int ampq_partition(int n, int n_edges, const int *edge_src, const int *edge_dst,
+                   const unsigned char *quantisable, int *group_of, int *n_groups);
+
+/* Performance-metric table of one group from layer shapes: c_out[p] = sum_l
+ * c_{l, Q[l + Lj*p]} with, per layer and format f,
+ *   AMPQ_GAIN_MAC     N C K delta[f] (linear), N C^2 delta[f] (BGEMM): the
+ *                     theoretical time gain of Sec. 2.3.2, delta[f] the time
+ *                     gained per multiply-accumulate in format f;
+ *   AMPQ_GAIN_MEMORY  C K delta[f] (linear), 0 (BGEMM): the memory gain of
+ *                     Sec. 2.3.3, delta[f] the bytes saved per stored parameter.
+ * N, C, K [Lj]; delta[F] (delta[0] = 0 for the baseline format).  Host pointers. */
+enum { AMPQ_GAIN_MAC = 0, AMPQ_GAIN_MEMORY = 1 };
+int ampq_gain_table(int gain_kind, int Lj, const int *layer_kind, const long long *N, const long long *C,
+                    const long long *K, const unsigned char *Q, int Pj, const double *delta, int F,
+                    double *c_out);
+
+/* The baseline strategies the paper compares with (Sec. 3.1): units (layers or
+ * groups) are switched to low precision one after the other in the order given
+ * while the loss-MSE budget holds, stopping at the first that does not fit.
+ * order = 0..L-1 is "Prefix"; a random permutation drawn by the caller is
+ * "Random".  d_low[u], c_low[u]: loss MSE and gain of unit u in low precision.
+ * chosen[u] = 1 for the units switched.  Host pointers. */
+int ampq_select_in_order(int L, const int *order, const double *d_low, const double *c_low, double budget,
+                         unsigned char *chosen, double *c_total, double *d_total);
+
 /* The paper has no counterpart of this call; it exists for callers that are
  * not allowed to allocate device memory: code that runs while another library
  * owns the device heap through its own pool, code in a phase where a device

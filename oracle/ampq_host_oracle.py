@@ -56,7 +56,8 @@ def partition(n, edges, quantisable):
     # separators: deleting the vertex cuts start from end
     seps = [v for v in range(n) if v == end or end not in _reach(succ, start, banned=v)]
     # order them along the paths: a reaches b  <=>  a comes first
-    seps.sort(key=lambda v: -len(_reach(succ, v) & set(seps)))
+    sepset = set(seps)
+    seps.sort(key=lambda v: -len(_reach(succ, v) & sepset))
     raw = []
     for u in range(n):
         reach = _reach(succ, u)

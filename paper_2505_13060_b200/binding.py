@@ -35,6 +35,7 @@ EXPORTS = [
     "ampq_define_group", "ampq_clear_groups", "ampq_group_costs", "ampq_budget_from_tau",
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
+    "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -83,6 +84,9 @@ def lib():
     L.ampq_stream_sample.argtypes = [vp, i, i, i, i, vp, vp, ll]
     L.ampq_stream_end.argtypes = [vp]
     L.ampq_fake_quant.argtypes = [vp, i, i, vp, ll, C.c_float, vp]
+    L.ampq_partition.argtypes = [i, i, vp, vp, vp, vp, ip]
+    L.ampq_gain_table.argtypes = [i, i, vp, vp, vp, vp, vp, i, vp, i, vp]
+    L.ampq_select_in_order.argtypes = [i, vp, vp, vp, C.c_double, vp, dp, dp]
     L.ampq_group_costs_table.argtypes = [vp, i, vp, i, vp, i, i, vp]
     L.ampq_budget_from_tau.argtypes = [C.c_double, vp, i, dp]
     L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
@@ -107,6 +111,52 @@ def budget_from_tau(tau: float, losses) -> float:
     if rc:
         raise AmpqError(rc)
     return out.value
+
+
+GAIN_MAC, GAIN_MEMORY = 0, 1
+
+
+def partition(n: int, edges, quantisable):
+    """Sequential sub-graphs of a model DAG (Algorithm 2).  Returns (group_of[n], J)."""
+    e = np.ascontiguousarray(np.asarray(edges, dtype=np.int32).reshape(-1, 2))
+    src, dst = np.ascontiguousarray(e[:, 0]), np.ascontiguousarray(e[:, 1])
+    q = np.ascontiguousarray(quantisable, dtype=np.uint8)
+    out = np.zeros(n, dtype=np.int32)
+    J = C.c_int()
+    rc = lib().ampq_partition(n, len(e), _np_ptr(src), _np_ptr(dst), _np_ptr(q), _np_ptr(out), C.byref(J))
+    if rc:
+        raise AmpqError(rc, "ampq_partition")
+    return out, J.value
+
+
+def gain_table(kind: int, layers, Q, delta) -> np.ndarray:
+    """layers: [(layer kind, N, C, K)] of one group; Q: [Lj, Pj]; delta: [F]."""
+    lk = np.ascontiguousarray([l[0] for l in layers], dtype=np.int32)
+    N, Cc, K = (np.ascontiguousarray([l[k] for l in layers], dtype=np.int64) for k in (1, 2, 3))
+    Q = np.asarray(Q, dtype=np.uint8)
+    Lj, Pj = Q.shape
+    Qf = np.ascontiguousarray(Q.T).reshape(-1)
+    dl = np.ascontiguousarray(delta, dtype=np.float64)
+    out = np.zeros(Pj)
+    rc = lib().ampq_gain_table(kind, Lj, _np_ptr(lk), _np_ptr(N), _np_ptr(Cc), _np_ptr(K), _np_ptr(Qf), Pj,
+                               _np_ptr(dl), dl.size, _np_ptr(out))
+    if rc:
+        raise AmpqError(rc, "ampq_gain_table")
+    return out
+
+
+def select_in_order(order, d_low, c_low, budget: float):
+    """Prefix / Random baselines: returns (chosen[L], c_total, d_total)."""
+    o = np.ascontiguousarray(order, dtype=np.int32)
+    d = np.ascontiguousarray(d_low, dtype=np.float64)
+    c = np.ascontiguousarray(c_low, dtype=np.float64)
+    ch = np.zeros(max(o.size, 1), dtype=np.uint8)
+    co, do = C.c_double(), C.c_double()
+    rc = lib().ampq_select_in_order(o.size, _np_ptr(o), _np_ptr(d), _np_ptr(c), budget, _np_ptr(ch), C.byref(co),
+                                    C.byref(do))
+    if rc:
+        raise AmpqError(rc, "ampq_select_in_order")
+    return ch[:o.size].copy(), co.value, do.value
 
 
 def group_costs_table(layer_ids, Q, d_layer) -> np.ndarray:

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libampq.so")
-SOURCES = ["ampq_kernels.cu", "ampq_lib.cu", "ampq_noalloc.cu", "ampq_select.cpp"]
+SOURCES = ["ampq_kernels.cu", "ampq_lib.cu", "ampq_noalloc.cu", "ampq_select.cpp", "ampq_graph.cpp"]
 HEADERS = ["ampq_device.h", "ampq_kernels.h", "ampq_select.h", os.path.join("..", "..", "include", "ampq.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -372,3 +372,53 @@ def test_full_size_llama70b_sampled_layers(ampq, orc):
             assert a["s_per_sample"].tobytes() == got["s_per_sample"].tobytes()
             assert a["d_meas_per_sample"].tobytes() == got["d_meas_per_sample"].tobytes()
     ctx.destroy()
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2])
+def test_format_budget_sweep_with_baseline_strategies(ampq, orc, fmt):
+    """The format / budget sweep: 32 scaled-down 7B-shaped blocks, 64 sub-graphs
+    (attention linears and MLP linears of every block), time gains drawn
+    uniformly in [0.5, 2] ms, budgets of 1, 5, 20 and 50 % of the all-low-precision
+    loss MSE.  The exact selection from the GPU tables equals the oracle's branch
+    and bound on its own tables; Prefix and Random (Sec. 3.1) pick the same units
+    from either table, stay within the budget and never gain more than the
+    integer program."""
+    specs = []
+    for b in range(32):
+        specs += synth.llama7b_block(64, prefix="b%d." % b)
+    lts = [synth.make_layer(s, "cuda", seed=5, layer=i) for i, s in enumerate(specs)]
+    ctx = _ctx(ampq, (0, fmt))
+    ids = _register(ampq, ctx, lts)
+    ctx.score()
+    refs = [oracle_layer(orc, lt, [fmt], threads=8) for lt in lts]
+    rng = np.random.default_rng(7)
+    tabs = []
+    for b in range(32):
+        for members in (list(range(7 * b, 7 * b + 4)), list(range(7 * b + 4, 7 * b + 7))):
+            Q = np.array([[0, 1]] * len(members), dtype=np.uint8)
+            c = np.array([0.0, rng.uniform(0.5, 2.0)])
+            ctx.define_group([ids[m] for m in members], Q, c)
+            tabs.append((members, Q, c))
+    perm = rng.permutation(len(tabs))
+    for mode, key in ((ampq.D_MODEL, "d_model"), (ampq.D_MEASURED, "d_meas")):
+        d_layer = np.array([r[key] for r in refs])
+        d_tabs = [orc.group_costs(m, Q, d_layer) for m, Q, _ in tabs]
+        gpu_tabs = [ctx.group_costs(j, mode) for j in range(len(tabs))]
+        all_low = float(np.sum(d_layer[:, 1]))
+        prev_c = -1.0
+        for frac in (0.01, 0.05, 0.2, 0.5):
+            want = orc.select_bnb([c for _, _, c in tabs], d_tabs, frac * all_low)
+            got = ctx.select(mode, frac * ctx.all_lowp_cost(mode, 1))
+            assert got[0].tolist() == want[0].tolist() and got[1] == want[1], (fmt, mode, frac)
+            assert got[1] >= prev_c   # the gain grows with the budget
+            prev_c = got[1]
+            for order in (np.arange(len(tabs)), perm):
+                from oracle import ampq_host_oracle as ho
+
+                ch, cs, ds = ampq.select_in_order(order, [t[1] for t in gpu_tabs], [c[1] for _, _, c in tabs],
+                                                  frac * ctx.all_lowp_cost(mode, 1))
+                wch, wcs, wds = ho.select_in_order(order.tolist(), [float(t[1]) for t in d_tabs],
+                                                   [float(c[1]) for _, _, c in tabs], frac * all_low)
+                assert ch.tolist() == wch and cs == wcs
+                assert ds <= frac * ctx.all_lowp_cost(mode, 1) and cs <= got[1]
+    ctx.destroy()

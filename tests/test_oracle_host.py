@@ -92,7 +92,8 @@ def test_partition_separators_against_path_counting():
         for u in range(n - 1):
             if not any(a == u for a, _ in edges):
                 edges.add((u, int(rng.integers(u + 1, n))))
-        edges = sorted(edges)
+        perm = rng.permutation(n)   # vertex numbers carry no order
+        edges = sorted((int(perm[a]), int(perm[b])) for a, b in edges)
         g, J = ho.partition(n, edges, [1] * n)
         down, up, order = _paths(n, edges)
         total = sum(up[v] for v in range(n) if down[v] == 1 and not any(b == v for _, b in edges))
