@@ -200,6 +200,21 @@ void orc_scales(int fmt, float amax, float *scale, float *inv_scale) {
     *inv_scale = inv;
 }
 
+/* Power-of-two scaling: the smallest power of two p with fmax * p >= amax, so
+ * that nothing saturates and z * (1/p) is exact; inv_scale = 1/p.  The neutral
+ * pair (1, 1) when amax = 0 or p (or 1/p) is not a normal fp32. */
+void orc_scales_pow2(int fmt, float amax, float *scale, float *inv_scale) {
+    double fmax = orc_fmax(fmt);
+    *scale = 1.0f;
+    *inv_scale = 1.0f;
+    if (!(amax > 0.0f) || isinf(amax)) return;
+    int k = -200;
+    while (ldexp(fmax, k) < (double)amax) ++k; /* plain search: exact comparisons in double */
+    if (k < -126 || k > 126) return;
+    *scale = (float)ldexp(1.0, k);
+    *inv_scale = (float)ldexp(1.0, -k);
+}
+
 /* Step 3 (codes only): q_k = encode_f( fl32( z_k * inv_scale ) ). */
 void orc_codes(int dtype, const void *values, long long n, int fmt, float inv_scale,
                unsigned char *codes) {

@@ -55,6 +55,8 @@ def lib():
         L.orc_amax.argtypes = [C.c_int, C.c_void_p, C.c_longlong]
         L.orc_scales.restype = None
         L.orc_scales.argtypes = [C.c_int, C.c_float, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.orc_scales_pow2.restype = None
+        L.orc_scales_pow2.argtypes = [C.c_int, C.c_float, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.orc_codes.restype = None
         L.orc_codes.argtypes = [C.c_int, C.c_void_p, C.c_longlong, C.c_int, C.c_float, C.c_void_p]
         L.orc_fake_quant.restype = None
@@ -121,9 +123,10 @@ def amax(values: np.ndarray) -> np.float32:
     return np.float32(lib().orc_amax(_dtype_of(v), _ptr(v), v.size))
 
 
-def scales(fmt: int, amax_value) -> tuple[np.float32, np.float32]:
+def scales(fmt: int, amax_value, pow2: bool = False) -> tuple[np.float32, np.float32]:
     s, i = C.c_float(), C.c_float()
-    lib().orc_scales(fmt, C.c_float(float(amax_value)), C.byref(s), C.byref(i))
+    fn = lib().orc_scales_pow2 if pow2 else lib().orc_scales
+    fn(fmt, C.c_float(float(amax_value)), C.byref(s), C.byref(i))
     return np.float32(s.value), np.float32(i.value)
 
 
@@ -158,7 +161,7 @@ def score_segment(values: np.ndarray, grads: np.ndarray, fmts, scale_list, inv_l
 
 
 def score_operand(values: np.ndarray, grads: np.ndarray, R: int, per_sample_values: bool,
-                  low_fmts, amax_preset=None, threads: int = 1):
+                  low_fmts, amax_preset=None, threads: int = 1, pow2: bool = False):
     """Steps 1-4 for one operand.
 
     values: per_sample_values -> [R, n] (sample r owns row r), else [n] shared by
@@ -172,7 +175,7 @@ def score_operand(values: np.ndarray, grads: np.ndarray, R: int, per_sample_valu
     a = amax(v) if amax_preset is None else np.float32(amax_preset)
     sc, iv = [], []
     for f in low_fmts:
-        s, i = scales(f, a)
+        s, i = scales(f, a, pow2)
         sc.append(s)
         iv.append(i)
     vv = v.reshape(R, -1) if per_sample_values else v.reshape(1, -1)

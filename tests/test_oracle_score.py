@@ -274,3 +274,31 @@ def test_fake_quant_pins(orc, dtype, f):
     s2, i2 = orc.scales(f, orc.amax(von))
     assert s2 == np.float32(0.25)
     assert np.array_equal(orc.fake_quant(von, f, s2, i2), von)
+
+
+@pytest.mark.parametrize("f", [1, 2])
+def test_power_of_two_scale_pins(orc, f):
+    """The power-of-two scale: a power of two, just large enough that amax does
+    not saturate (fmax*p >= amax > fmax*p/2, checked in rational arithmetic),
+    equal to the amax scale when amax is fmax times a power of two, neutral for 0
+    and for magnitudes whose scale is not a normal fp32."""
+    fmax = Fraction(orc.fmax(f))
+    rng = np.random.default_rng(8)
+    for a in list(np.exp(rng.uniform(-60, 60, 200)).astype(np.float32)) + [np.float32(1.0), np.float32(448.0)]:
+        sc, iv = orc.scales(f, a, pow2=True)
+        m, e = np.frexp(float(sc))
+        assert m == 0.5 and float(sc) * float(iv) == 1.0
+        assert fmax * Fraction(float(sc)) >= Fraction(float(a)) > fmax * Fraction(float(sc)) / 2
+    for k in (-20, 0, 13):
+        a = np.float32(float(fmax) * 2.0 ** k)
+        assert orc.scales(f, a, pow2=True) == orc.scales(f, a) == (np.float32(2.0 ** k), np.float32(2.0 ** -k))
+        up = np.nextafter(a, np.float32(np.inf))
+        assert orc.scales(f, up, pow2=True)[0] == np.float32(2.0 ** (k + 1))
+    assert orc.scales(f, 0.0, pow2=True) == (1.0, 1.0)
+    assert orc.scales(f, np.float32(1e-44), pow2=True) == (1.0, 1.0)
+    # with a power-of-two scale the scaled value is exact, so the codes of z and of 4z agree
+    v = (rng.standard_normal(1000) * 3).astype(np.float32)
+    a, sc, iv, seg = orc.score_operand(v, np.ones(1000, np.float32), 1, False, [f], pow2=True)
+    a4, sc4, iv4, seg4 = orc.score_operand(4 * v, np.ones(1000, np.float32), 1, False, [f], pow2=True)
+    assert sc4[0] == 4 * sc[0] and seg4[0, 1] == 16 * seg[0, 1]
+    assert np.array_equal(orc.codes(v, f, iv[0]), orc.codes(4 * v, f, iv4[0]))
