@@ -112,6 +112,24 @@ int ampq_bind_operand(ampq_ctx *ctx, int layer_id, int operand, int dtype, int m
  * negative amax removes the preset. */
 int ampq_set_amax(ampq_ctx *ctx, int layer_id, int operand, float amax);
 
+/* How the per-tensor scale is formed from amax (default AMPQ_SCALE_AMAX):
+ *   AMPQ_SCALE_AMAX  scale = fl32(amax/fmax_f), inv = fl32(fmax_f/amax)
+ *   AMPQ_SCALE_POW2  scale = the smallest power of two p with fmax_f*p >= amax,
+ *                    inv = 1/p: nothing saturates and z*inv is exact; (1,1)
+ *                    when amax = 0 or p is not a normal fp32.
+ * Applies to ampq_score, ampq_stream_sample and ampq_fake_quant. */
+enum { AMPQ_SCALE_AMAX = 0, AMPQ_SCALE_POW2 = 1 };
+int ampq_set_scale_mode(ampq_ctx *ctx, int mode);
+
+/* Only the first step of ampq_score: amax of every bound operand of every fully
+ * bound layer (preset ones keep their preset), asynchronously on the stream.
+ * ampq_get_amax (synchronises) then gives amax[2] of a layer; it also works
+ * after ampq_score.  Meant for calibration split over several processes by
+ * sample: each measures its own samples, the maxima are combined outside (a
+ * MAX all-reduce), set with ampq_set_amax, and then every process scores. */
+int ampq_measure_amax(ampq_ctx *ctx);
+int ampq_get_amax(ampq_ctx *ctx, int layer_id, float *amax);
+
 /* Scores every layer whose two operands are bound (Algorithm 1 step 2, the
  * per-element part), asynchronously on the context's stream:
  *   amax_t = max_k |z_k| per tensor; per format f: scale = fl32(amax/fmax_f),

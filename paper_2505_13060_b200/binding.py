@@ -22,6 +22,7 @@ FMT_BASE, FMT_E4M3, FMT_E5M2 = 0, 1, 2
 LINEAR, BGEMM = 0, 1
 D_MODEL, D_MEASURED = 0, 1
 MEM_DEVICE, MEM_HOST = 0, 1
+SCALE_AMAX, SCALE_POW2 = 0, 1
 
 OK = 0
 ERR_INVALID, ERR_ALIGN, ERR_STATE, ERR_CUDA = -1, -2, -3, -4
@@ -36,6 +37,7 @@ EXPORTS = [
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
+    "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -84,6 +86,9 @@ def lib():
     L.ampq_stream_sample.argtypes = [vp, i, i, i, i, vp, vp, ll]
     L.ampq_stream_end.argtypes = [vp]
     L.ampq_fake_quant.argtypes = [vp, i, i, vp, ll, C.c_float, vp]
+    L.ampq_set_scale_mode.argtypes = [vp, i]
+    L.ampq_measure_amax.argtypes = [vp]
+    L.ampq_get_amax.argtypes = [vp, i, vp]
     L.ampq_partition.argtypes = [i, i, vp, vp, vp, vp, ip]
     L.ampq_gain_table.argtypes = [i, i, vp, vp, vp, vp, vp, i, vp, i, vp]
     L.ampq_select_in_order.argtypes = [i, vp, vp, vp, C.c_double, vp, dp, dp]
@@ -255,6 +260,17 @@ class Context:
 
     def set_amax(self, layer_id: int, operand: int, amax: float):
         self._check(lib().ampq_set_amax(self._h, layer_id, operand, amax))
+
+    def set_scale_mode(self, mode: int):
+        self._check(lib().ampq_set_scale_mode(self._h, mode))
+
+    def measure_amax(self):
+        self._check(lib().ampq_measure_amax(self._h))
+
+    def get_amax(self, layer_id: int) -> np.ndarray:
+        out = np.zeros(2, np.float32)
+        self._check(lib().ampq_get_amax(self._h, layer_id, _np_ptr(out)))
+        return out
 
     def score(self):
         self._check(lib().ampq_score(self._h))

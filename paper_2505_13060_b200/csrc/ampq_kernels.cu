@@ -204,9 +204,13 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
 
 // scale = fl32(amax / fmax), inv = fl32(fmax / amax), IEEE divisions; the
 // neutral pair (1, 1) when amax is 0 or fmax/amax is not a finite fp32.
+// pow2 mode: scale = the smallest power of two p with fmax * p >= amax, inv =
+// 1/p.  With fmax = 1.75 * 2^ef and amax = m * 2^ea (1 <= m < 2) that is
+// 2^(ea - ef) when m <= 1.75 and 2^(ea - ef + 1) otherwise, read off the bits;
+// neutral when p or 1/p is not a normal fp32.
 __global__ void scales_kernel(int T, int fmask, const unsigned* __restrict__ amax_bits,
                               float* __restrict__ scales, int* __restrict__ tensor_flags,
-                              LaunchStatus* status) {
+                              LaunchStatus* status, int pow2) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
     unsigned bits = amax_bits[t];
@@ -220,7 +224,15 @@ __global__ void scales_kernel(int T, int fmask, const unsigned* __restrict__ ama
         if (!(fmask & f)) continue;
         float fmax = (f == kMaskE4M3) ? 448.0f : 57344.0f;
         float scale = 1.0f, inv = 1.0f;
-        if (!bad && amax > 0.0f) {
+        if (!bad && amax > 0.0f && pow2) {
+            const int ef = (f == kMaskE4M3) ? 8 : 15;
+            const int field = (int)(bits >> 23);  // 0 for a subnormal amax: far below the range anyway
+            const int k = field - 127 - ef + ((bits & 0x7FFFFFu) > 0x600000u ? 1 : 0);
+            if (field > 0 && k >= -126 && k <= 126) {
+                scale = __uint_as_float((unsigned)(k + 127) << 23);
+                inv = __uint_as_float((unsigned)(127 - k) << 23);
+            }
+        } else if (!bad && amax > 0.0f) {
             float i = __fdiv_rn(fmax, amax);
             if (i <= 3.402823466e+38f) {
                 inv = i;
@@ -876,9 +888,9 @@ cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, 
 }
 
 cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
-                          LaunchStatus* status, cudaStream_t st) {
+                          LaunchStatus* status, cudaStream_t st, int pow2) {
     if (T <= 0) return cudaSuccess;
-    scales_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, fmask, amax_bits, scales, tensor_flags, status);
+    scales_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, fmask, amax_bits, scales, tensor_flags, status, pow2);
     return cudaGetLastError();
 }
 

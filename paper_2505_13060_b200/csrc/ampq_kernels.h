@@ -18,8 +18,9 @@ cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, Lau
                              cudaStream_t st);
 cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                         unsigned* amax_bits, cudaStream_t st);
+// pow2 = 1: power-of-two scales instead of amax / fmax.
 cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
-                          LaunchStatus* status, cudaStream_t st);
+                          LaunchStatus* status, cudaStream_t st, int pow2 = 0);
 // One launch per element type (0 = fp32, 1 = bf16) and sample-group size rb =
 // 1..kMaxRB, each with its own tile table.
 // Tiles hold 2^tile_shift elements; the persistent grid has at most max_ctas CTAs

@@ -102,6 +102,8 @@ struct ampq_ctx {
     int slot_of_fmt[1 + kMaxLow] = {-1, 0, -1};  // user format index -> internal low slot
     std::vector<LayerRec> layers;
     std::vector<Group> groups;
+    int scale_pow2 = 0;    // AMPQ_SCALE_POW2: power-of-two scales
+    bool amax_ready = false;  // ampq_measure_amax (or a score) has filled the amax mirror
     bool dirty = true;     // bindings changed since the tables were built
     bool scored = false;   // a score has been issued
     bool pending = false;  // its results have not been synchronised yet
@@ -399,6 +401,25 @@ int group_costs_impl(ampq_ctx* ctx, const Group& g, int d_mode, double* d_out) {
     return AMPQ_OK;
 }
 
+// Common start of a full pass: wait for the previous read-back, end any
+// streaming pass, rebuild and upload the tables when the bindings changed.
+int prepare_tables(ampq_ctx* ctx) {
+    int rc;
+    if (ctx->pending) {  // the previous pass's read-back still owns the pinned mirrors
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        ctx->pending = false;
+    }
+    ctx->streaming = false;
+    if (ctx->dirty) {
+        ctx->scored = false;
+        ctx->amax_ready = false;
+        if ((rc = build_tables(ctx))) return rc;
+        if ((rc = upload_tables(ctx))) return rc;
+        ctx->dirty = false;
+    }
+    return AMPQ_OK;
+}
+
 // Per-layer combine and the asynchronous read-back of every small result.
 int combine_and_read_back(ampq_ctx* ctx, int T, int L, int S) {
     const int nacc = ctx->F;
@@ -428,7 +449,7 @@ int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, int dtype, const void* v
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
     AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, st), "job_prepare");
     AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st), "amax");
-    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, ctx->d_status.p, st), "scales");
+    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, ctx->d_status.p, st, ctx->scale_pow2), "scales");
     return AMPQ_OK;
 }
 
@@ -567,22 +588,59 @@ int ampq_set_amax(ampq_ctx* ctx, int layer_id, int operand, float amax) {
     return AMPQ_OK;
 }
 
+int ampq_set_scale_mode(ampq_ctx* ctx, int mode) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    if (mode != AMPQ_SCALE_AMAX && mode != AMPQ_SCALE_POW2) return fail(ctx, AMPQ_ERR_INVALID, "unknown scale mode");
+    ctx->scale_pow2 = mode == AMPQ_SCALE_POW2 ? 1 : 0;
+    ctx->scored = false;
+    return AMPQ_OK;
+}
+
+int ampq_measure_amax(ampq_ctx* ctx) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
+    int rc;
+    if ((rc = prepare_tables(ctx))) return rc;
+    ctx->scored = false;
+    const int T = (int)ctx->tens.size();
+    cudaStream_t st = ctx->stream;
+    ctx->launches = 0;
+    ctx->ev_valid = false;
+    if ((rc = stage_host_operands(ctx))) return rc;
+    if (T > 0) {
+        AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
+        AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
+        ctx->launches = ctx->namax_tiles > 0 ? 2 : 1;
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
+    }
+    ctx->amax_ready = true;
+    ctx->pending = T > 0;
+    return AMPQ_OK;
+}
+
+int ampq_get_amax(ampq_ctx* ctx, int layer_id, float* amax) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (!amax) return fail(ctx, AMPQ_ERR_INVALID, "null output");
+    if (!ctx->amax_ready || ctx->dirty) return fail(ctx, AMPQ_ERR_STATE, "no amax has been measured for the current bindings");
+    DeviceGuard g(ctx->device);
+    if (ctx->pending) {
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        ctx->pending = false;
+    }
+    const LayerRec& l = ctx->layers[layer_id];
+    if (l.scored < 0) return fail(ctx, AMPQ_ERR_STATE, "layer has an unbound operand");
+    for (int k = 0; k < 2; ++k) std::memcpy(&amax[k], &ctx->h_amax_bits.p[l.op[k].tensor], sizeof(float));
+    return AMPQ_OK;
+}
+
 int ampq_score(ampq_ctx* ctx) {
     if (!ctx) return AMPQ_ERR_INVALID;
     DeviceGuard g(ctx->device);
     if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
     int rc;
-    if (ctx->pending) {  // the previous score's read-back still owns the pinned mirrors
-        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
-        ctx->pending = false;
-    }
-    ctx->streaming = false;  // a full score ends any streaming pass
-    if (ctx->dirty) {
-        ctx->scored = false;
-        if ((rc = build_tables(ctx))) return rc;
-        if ((rc = upload_tables(ctx))) return rc;
-        ctx->dirty = false;
-    }
+    if ((rc = prepare_tables(ctx))) return rc;
     const int T = (int)ctx->tens.size(), L = (int)ctx->lay.size(), S = (int)ctx->segs.size();
     const int nacc = ctx->F;  // S plus one D per low-precision format
     cudaStream_t st = ctx->stream;
@@ -600,7 +658,7 @@ int ampq_score(ampq_ctx* ctx) {
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
-        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st), "scales");
+        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         for (int c = 0; c < kScoreClasses; ++c) {
@@ -618,6 +676,7 @@ int ampq_score(ampq_ctx* ctx) {
         }
     }
     ctx->scored = true;
+    ctx->amax_ready = true;
     ctx->pending = T > 0;
     return AMPQ_OK;
 }

@@ -70,3 +70,45 @@ def select_from_table(binding, table: np.ndarray, F: int, groups, d_mode: int, b
         c_tabs.append(np.asarray(c, dtype=np.float64))
         d_tabs.append(binding.group_costs_table(layer_ids, Q, d_layer))
     return binding.select_tables(c_tabs, d_tabs, budget)
+
+
+# ---------------------------------------------------------------------------
+# Sample-sharded calibration: every rank holds the same layers but only its own
+# calibration samples.  Two small exchanges: the per-tensor amax (MAX) between
+# the amax pass and the scoring pass, and the per-layer rows (a mean over all
+# samples, Sec. 2.2) afterwards.
+
+def reduce_amax(local_amax, group=None, device=None) -> np.ndarray:
+    """``local_amax``: [L, 2] float32 from ``Context.get_amax`` on this rank's
+    samples.  Returns the element-wise maximum over all ranks (exact)."""
+    import torch
+    import torch.distributed as dist
+
+    a = np.ascontiguousarray(local_amax, dtype=np.float32)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        t = torch.from_numpy(a.copy())
+        if device is not None:
+            t = t.to(device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
+        a = t.cpu().numpy()
+    return a
+
+
+def merge_sample_rows(local_table, R_local: int, group=None, device=None) -> np.ndarray:
+    """``local_table``: [L, 1 + 2F] rows (``layer_row``) computed over this rank's
+    ``R_local`` samples.  Every entry is a mean over samples, so the value over
+    all samples is the R-weighted mean over ranks: one SUM all-reduce of
+    [R_local * rows | R_local]."""
+    import torch
+    import torch.distributed as dist
+
+    tab = np.ascontiguousarray(local_table, dtype=np.float64)
+    if not (dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1):
+        return tab
+    buf = np.concatenate([(tab * float(R_local)).reshape(-1), [float(R_local)]])
+    t = torch.from_numpy(buf)
+    if device is not None:
+        t = t.to(device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    out = t.cpu().numpy()
+    return out[:-1].reshape(tab.shape) / out[-1]

@@ -63,10 +63,17 @@ def worker(rank, world, port, out):
         for frac in (0.05, 0.5):
             p, c, d = shard.select_from_table(binding, table, F, groups, mode, frac * all_low)
             res["%d_%g" % (mode, frac)] = [p.tolist(), c, d]
+    # sample-sharded exchanges: MAX of amax, R-weighted mean of the rows
+    a = np.array([[1.0 + rank, 5.0 - rank], [0.25, 0.25 * (rank + 1)]], np.float32)
+    amax = shard.reduce_amax(a)
+    R_local = 3 if rank == 0 else 5
+    rows = np.array([[1.0, 0.0, 2.0, 0.0, 4.0], [8.0, 0.0, 1.0, 0.0, 0.5]]) * (rank + 1)
+    merged = shard.merge_sample_rows(rows, R_local)
     dist.barrier()
     dist.destroy_process_group()
     with open(os.path.join(out, "rank%d.json" % rank), "w") as f:
-        json.dump({"owner": owner.tolist(), "mine": mine, "table": table.tolist(), "res": res}, f)
+        json.dump({"owner": owner.tolist(), "mine": mine, "table": table.tolist(), "res": res,
+                   "amax": amax.tolist(), "merged": merged.tolist()}, f)
 
 
 def test_two_ranks_agree_with_one_process(tmp_path, ampq, orc):
@@ -79,6 +86,10 @@ def test_two_ranks_agree_with_one_process(tmp_path, ampq, orc):
     for p in procs:
         assert p.wait(timeout=300) == 0
     got = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in range(2)]
+    # sample-sharded exchanges: element-wise maximum; (3*rows + 5*2*rows)/8
+    assert got[0]["amax"] == got[1]["amax"] == [[2.0, 5.0], [0.25, 0.5]]
+    base = np.array([[1.0, 0.0, 2.0, 0.0, 4.0], [8.0, 0.0, 1.0, 0.0, 0.5]])
+    assert got[0]["merged"] == got[1]["merged"] == (base * 13.0 / 8.0).tolist()
     # both ranks hold the same table and the same plans, bit for bit
     assert got[0]["table"] == got[1]["table"] and got[0]["res"] == got[1]["res"]
     assert got[0]["owner"] == got[1]["owner"]
