@@ -422,3 +422,38 @@ def test_format_budget_sweep_with_baseline_strategies(ampq, orc, fmt):
                 assert ch.tolist() == wch and cs == wcs
                 assert ds <= frac * ctx.all_lowp_cost(mode, 1) and cs <= got[1]
     ctx.destroy()
+
+
+def test_operand_with_more_than_2_31_elements(ampq, orc):
+    """64-bit indexing: one bf16 operand of 2^31 + 2^20 + 777 elements (4.3 GB,
+    as much again for its gradient), built as repeats of one 2^20-element block
+    plus a ragged piece of it, so that the sums are the block's sums (from the
+    oracle) times the repeat count plus those of the piece."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12e9:
+        pytest.skip("needs 12 GB of free device memory")
+    nb, reps, tail = 1 << 20, 2049, 777
+    g = torch.Generator(device="cuda").manual_seed(17)
+    vb = torch.empty(nb, dtype=torch.bfloat16, device="cuda").normal_(0, 1, generator=g)
+    gb = torch.empty(nb, dtype=torch.bfloat16, device="cuda").normal_(0, 1, generator=g) * 1e-3
+    vb[12345] = 37.0   # the amax sits inside the block, hence in every repeat
+    n = nb * reps + tail
+    v = torch.cat([vb.repeat(reps), vb[:tail]])
+    gr = torch.cat([gb.repeat(reps), gb[:tail]])
+    assert v.numel() == n > 2 ** 31
+    ctx = _ctx(ampq, (0, E4M3))
+    lid = ctx.register_layer(ampq.LINEAR, "huge", 1)
+    ctx.bind_operand(lid, 0, ampq.BF16, v.data_ptr(), n, True, gr.data_ptr(), n)
+    ctx.bind_operand(lid, 1, ampq.BF16, 0, 0, False, 0, 0)
+    ctx.score()
+    got = ctx.get_operand(lid, 0)[0]
+    hv, hg = synth.to_numpy(vb), synth.to_numpy(gb)
+    a, sc, iv, seg_block = orc.score_operand(hv, hg, 1, False, [E4M3])
+    seg_tail = orc.score_segment(hv[:tail], hg[:tail], [E4M3], sc, iv)
+    assert ctx.get_layer(lid)["amax"][0] == a == np.float32(37.0)
+    assert_close(got, reps * seg_block[0] + seg_tail, "2^31+ elements [S, D]", tol=1e-9)
+    # the last element really is read: moving the amax there changes the scale
+    v[n - 1] = 100.0
+    ctx.score()
+    assert ctx.get_layer(lid)["amax"][0] == np.float32(100.0)
+    ctx.destroy()

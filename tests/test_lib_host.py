@@ -115,3 +115,17 @@ def test_select_edge_cases(ampq):
     a = ampq.select_tables(c, d, 0.4 * hi)
     b = ampq.select_tables([2.5 * t + 1.0 for t in c], d, 0.4 * hi)
     assert a[0].tolist() == b[0].tolist()
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/ampq.h compiles as C99 and as C++ on its own (no CUDA, no torch
+    types), and a C program can name every declared entry point."""
+    import subprocess
+
+    hdr = os.path.join(ROOT, "include", "ampq.h")
+    names = _declared_symbols()
+    src = tmp_path / "use.c"
+    src.write_text('#include "%s"\nvoid *table[] = {%s};\nint main(void) { return AMPQ_OK; }\n'
+                   % (hdr, ", ".join("(void *)%s" % n for n in names)))
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-c", str(src), "-o", str(tmp_path / "use.o")])
+    subprocess.check_call(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr])
