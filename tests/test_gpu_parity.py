@@ -451,7 +451,7 @@ def test_operand_with_more_than_2_31_elements(ampq, orc):
     a, sc, iv, seg_block = orc.score_operand(hv, hg, 1, False, [E4M3])
     seg_tail = orc.score_segment(hv[:tail], hg[:tail], [E4M3], sc, iv)
     assert ctx.get_layer(lid)["amax"][0] == a == np.float32(37.0)
-    assert_close(got, reps * seg_block[0] + seg_tail, "2^31+ elements [S, D]", tol=1e-9)
+    assert_close(got, reps * seg_block[0] + seg_tail, "2^31+ elements [S, D]", tol=1e-6)   # one lost 8 KiB chunk would be 2e-6
     # the last element really is read: moving the amax there changes the scale
     v[n - 1] = 100.0
     ctx.score()
