@@ -59,8 +59,11 @@ def parse_args():
                     help="distinct 70B-shaped blocks held on the device (7.68 GB each)")
     ap.add_argument("--blocks", type=int, default=NUM_BLOCKS, help="blocks scored per step (the config has 80)")
     ap.add_argument("--formats", default="e4m3", choices=["e4m3", "e5m2", "both"])
-    ap.add_argument("--workload", default="llama70b", choices=["llama70b", "llama7b"],
-                    help="llama70b is the benchmark; llama7b (3.2 GB per block) is the small case for profiler captures")
+    ap.add_argument("--workload", default="llama70b", choices=["llama70b", "llama7b", "attention"],
+                    help="llama70b is the benchmark; llama7b (3.2 GB per block) and attention (the two BGEMMs of one "
+                         "attention layer per block, 2.55 GB) are side measurements, never the headline")
+    ap.add_argument("--causal", action="store_true",
+                    help="attention workload: declare the softmax operand causal so that its zero triangle is not read")
     ap.add_argument("--layers", default="",
                     help="comma-separated subset of a block's layers (q,k,v,o,gate,up,down); a small case of the "
                          "same kernels for profiler captures, never the benchmark")
@@ -245,7 +248,8 @@ def workload_specs(workload: str, layers: str = ""):
     """Layer specs of one block of the named workload (optionally a subset of its layers)."""
     from paper_2505_13060_b200 import synth
 
-    specs = synth.llama70b_block() if workload == "llama70b" else synth.llama7b_block()
+    specs = {"llama70b": synth.llama70b_block, "llama7b": synth.llama7b_block,
+             "attention": synth.attention_bgemm}[workload]()
     if layers:
         keep = layers.split(",")
         specs = [sp for sp in specs if sp.name in keep]
@@ -254,9 +258,11 @@ def workload_specs(workload: str, layers: str = ""):
     return specs
 
 
-def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int):
+def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int, causal: bool = False):
     """Registers `blocks` blocks of `specs` in ctx.  Block b is bound to device
     slot b mod nres; each slot is a full block of distinct random tensors.
+    With `causal`, causal-softmax operands are declared triangular and only the
+    bytes on or left of the diagonal count as scored.
     Returns (slots, layer ids, scored bytes of one score)."""
     import torch
 
@@ -274,6 +280,12 @@ def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int):
             ampq.bind_layer_tensors(ctx, lid, slots[b % nres][i])
             ids.append(lid)
             scored_bytes += sp.scored_bytes()
+            for k, op in enumerate((sp.op0, sp.op1)):
+                if causal and op.dist == "causal_softmax":
+                    T = op.shape[-1]
+                    ctx.set_causal(lid, k, T)
+                    es = slots[b % nres][i].values[k].element_size()
+                    scored_bytes -= 2 * es * (op.numel // (T * T)) * (T * (T - 1) // 2)   # the triangle not read
     return slots, ids, scored_bytes
 
 
@@ -304,7 +316,7 @@ def run_b200(args):
     stream = torch.cuda.Stream(device=dev)
     ctx = ampq.Context(local_rank, stream.cuda_stream)
     ctx.set_formats(fmts)
-    slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev, seed=100 + rank)
+    slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev, seed=100 + rank, causal=args.causal)
     value_bytes = args.blocks * sum(sp.value_bytes() for sp in specs)
     ctx.set_timing(True)
 
@@ -424,8 +436,8 @@ def run_b200(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
-                "tokens_per_sample": specs[0].op0.shape[1], "operand_dtype": "bf16", "formats": args.formats,
+                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else "") + ("[causal]" if args.causal else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
+                "tokens_per_sample": specs[0].op0.shape[-2], "operand_dtype": "bf16", "formats": args.formats,
                 "scored_bytes_per_step_per_gpu": scored_bytes, "resident_blocks": nres,
                 "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block" % (nres, block_gb),
                 "l2": "inputs larger than L2 (%.1f GB resident, 126 MB L2)" % (nres * block_gb),

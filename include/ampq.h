@@ -112,6 +112,19 @@ int ampq_bind_operand(ampq_ctx *ctx, int layer_id, int operand, int dtype, int m
  * negative amax removes the preset. */
 int ampq_set_amax(ampq_ctx *ctx, int layer_id, int operand, float amax);
 
+/* Declares that every sample slice of a per-sample operand is a stack of T x T
+ * matrices (the last two dimensions) whose entries right of the diagonal are
+ * EXACTLY zero, as in a causal softmax.  Such entries add nothing to amax, S or
+ * D_f whatever their gradient holds, so the library does not read them (about
+ * half the bytes of the operand and of its gradient).  Taken up when T is a
+ * power of two in [64, 32768], a sample slice is a whole number of matrices and
+ * the slices are 16-byte aligned; otherwise the operand is scored in full, with
+ * the same result.  The declaration is a promise: if the triangle is not zero,
+ * some of its entries (those sharing a 16-byte vector with the diagonal) are
+ * still scored and the rest are not, so the result is neither the dense one nor
+ * that of the zeroed operand.  T = 0 removes the declaration. */
+int ampq_set_causal(ampq_ctx *ctx, int layer_id, int operand, long long T);
+
 /* How the per-tensor scale is formed from amax (default AMPQ_SCALE_AMAX):
  *   AMPQ_SCALE_AMAX  scale = fl32(amax/fmax_f), inv = fl32(fmax_f/amax)
  *   AMPQ_SCALE_POW2  scale = the smallest power of two p with fmax_f*p >= amax,

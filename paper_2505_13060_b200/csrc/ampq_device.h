@@ -30,7 +30,9 @@ static_assert((1 << kMinTileShift) % kSubElems == 0, "a scoring tile is a whole 
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
 constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
-constexpr int kScoreClasses = 2 * kMaxRB;  // scoring launches of one score: element type x samples per read
+constexpr int kScoreClasses = 2 * kMaxRB + 2;  // scoring launches of one score: element type x samples per read,
+                                               // plus one class per element type for causal (triangular) operands
+constexpr int kMinCausalShift = 6, kMaxCausalShift = 15;  // T between 64 and 32768
 
 // internal low-precision slots: bit 0 = E4M3, bit 1 = E5M2.  With both present
 // slot 0 is E4M3 and slot 1 is E5M2; with one present it is slot 0.
@@ -52,7 +54,8 @@ struct Tensor {
     int rgroups;             // unused by the kernels (kept for table dumps): ceil(R / kMaxRB) or 1
     int seg_base;            // index of segment (this tensor, r = 0) in the segment outputs
     float amax_preset;       // >= 0: use instead of measuring
-    int pad;
+    int causal_shift;        // > 0: segments are stacks of T x T matrices, T = 2^causal_shift, whose strictly
+                             // upper triangles are exactly zero and are not read; 0: dense
 };
 
 // One segment = (tensor, sample): its partial slots are contiguous.

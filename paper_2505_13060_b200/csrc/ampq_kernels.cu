@@ -112,6 +112,15 @@ __device__ __forceinline__ int find_tensor(const long long* __restrict__ begin, 
     return *s_slot;
 }
 
+// Causal operands: element e of a segment sits in row (e >> shift) of a stack of
+// T x T matrices (T = 2^shift), at column e & (T-1) of matrix row
+// (e >> shift) & (T-1); everything right of the diagonal is exactly zero and is
+// never read.  Reads go in whole 16-byte vectors: matrix row i keeps its first
+// i / kPerVec + 1 vectors.
+__device__ __forceinline__ int causal_row_vectors(long long row, int shift, int per_vec) {
+    return (int)(row & ((1 << shift) - 1)) / per_vec + 1;
+}
+
 // ---------------------------------------------------------------------------
 // amax
 
@@ -142,7 +151,39 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
     const int es = tn.dtype == 0 ? 4 : 2;
     const char* base = reinterpret_cast<const char*>(tn.values) + first * es;
     unsigned m = 0;  // fp32 bit pattern of the running max |x|
-    if ((reinterpret_cast<uintptr_t>(base) & 15) == 0) {
+    if (tn.causal_shift > 0) {
+        // triangular operand (16-byte aligned, whole rows per tile): warp w takes
+        // rows w, w + 8, ... of the tile and its lanes stride over the vectors the
+        // row keeps, four loads in flight per lane
+        const int per = 16 / es;
+        const int shift = tn.causal_shift;
+        const int nrows = n >> shift;
+        const long long row0 = first >> shift;
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        for (int r = warp; r < nrows; r += kThreads / 32) {
+            const int nv = causal_row_vectors(row0 + r, shift, per);
+            const uint4* vp = reinterpret_cast<const uint4*>(base + ((long long)r << shift) * es);
+            for (int c = lane; c < nv; c += 32 * 4) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    v[u] = c + 32 * u < nv ? ld_stream_v4(vp + c + 32 * u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (tn.dtype == 0) {
+                            m = max(m, w[k] & 0x7FFFFFFFu);
+                        } else {
+                            m = max(m, (w[k] & 0x7FFFu) << 16);
+                            m = max(m, w[k] & 0x7FFF0000u);
+                        }
+                    }
+                }
+            }
+        }
+    } else if ((reinterpret_cast<uintptr_t>(base) & 15) == 0) {
         const int per = 16 / es;
         const int nvec = n / per;
         const uint4* vp = reinterpret_cast<const uint4*>(base);
@@ -477,6 +518,55 @@ __device__ __forceinline__ void score_direct(const char* vbase, const char* cons
     }
 }
 
+// One tile of a causal operand (one sample per read): whole matrix rows, of
+// which only the vectors on or left of the diagonal are read -- straight from
+// global memory, because a row's kept part is one short contiguous run and the
+// ring would need one bulk copy per row and stream (the copy rate, not the
+// bytes, then sets the pace).  Warp w takes rows w, w + 8, ... of the tile;
+// its lanes stride over the row's vectors with kU loads per stream in flight.
+template <int DT, int FMASK>
+__device__ __forceinline__ void score_causal_rows(const char* vbase, const char* gbase, int n, long long row0,
+                                                  int shift, const float2 (&inv2)[2], const float2 (&nsc2)[2],
+                                                  double (&acc64)[1][Fm<FMASK>::kAcc]) {
+    using E = Elem<DT>;
+    constexpr int NACC = Fm<FMASK>::kAcc;
+    constexpr int NP = E::kPerVec / 2;
+    constexpr int kU = 4;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nrows = n >> shift;
+    Acc<NACC> acc[1];
+#pragma unroll
+    for (int a = 0; a < NACC; ++a) acc[0].v[a] = make_float2(0.0f, 0.0f);
+    int since_flush = 0;
+    for (int r = warp; r < nrows; r += kConsumers / 32) {
+        const int nv = causal_row_vectors(row0 + r, shift, E::kPerVec);
+        const uint4* vp = reinterpret_cast<const uint4*>(vbase + ((long long)r << shift) * E::kBytes);
+        const uint4* gp = reinterpret_cast<const uint4*>(gbase + ((long long)r << shift) * E::kBytes);
+        for (int c = lane; c < nv; c += 32 * kU) {
+            uint4 v[kU], g[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const bool live = c + 32 * u < nv;
+                v[u] = live ? ld_stream_v4(vp + c + 32 * u) : make_uint4(0, 0, 0, 0);
+                g[u] = live ? ld_stream_v4(gp + c + 32 * u) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                float2 z[NP], gg[1][NP];
+                E::unpack(v[u], z);
+                E::unpack(g[u], gg[0]);
+                accumulate_pairs<FMASK, 1, NP>(z, gg, inv2, nsc2, acc);
+            }
+            since_flush += kU * NP;
+            if (since_flush + kU * NP > kFlushTerms) {  // at most kFlushTerms terms per fp32 lane
+                flush_acc<NACC, 1>(acc, acc64);
+                since_flush = 0;
+            }
+        }
+    }
+    flush_acc<NACC, 1>(acc, acc64);
+}
+
 // Geometry of the ring for RB gradient streams per value stream.  The
 // compile-time knobs exist for tuning builds; the defaults are what was
 // measured best on B200.
@@ -561,7 +651,7 @@ struct TileGeom {
     int r0, n;
 };
 
-template <int RB>
+template <int RB, bool CAUSAL>
 __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, int tile_shift) {
     TileGeom q;
     int i;  // value tile within the segment
@@ -578,6 +668,19 @@ __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, i
         i = local;
         q.r0 = (tn.R / kMaxRB) * kMaxRB;
         q.voff = (long long)i << tile_shift;
+    }
+    if (CAUSAL && 2 * tn.causal_shift > tile_shift) {
+        // A T x T triangular matrix spans P = T^2 / tile tiles whose work grows with
+        // their position k in the matrix (tile k holds rows whose kept prefix is
+        // about k/P of a row).  A persistent CTA walks the tiles with a fixed
+        // stride, which for common P would always land it on the same k; rotating k
+        // by a hash of the matrix index gives every CTA every k.  The partial slot
+        // follows the tile's true position, so the sums do not change.
+        const int lp = 2 * tn.causal_shift - tile_shift;
+        const unsigned m = (unsigned)i >> lp, k = (unsigned)i & ((1u << lp) - 1u);
+        const unsigned rot = (m * 0x9E3779B1u) >> (32 - lp);
+        i = (int)((m << lp) | ((k + rot) & ((1u << lp) - 1u)));
+        q.voff = (long long)q.r0 * tn.seg_len + ((long long)i << tile_shift);
     }
     q.goff = (long long)i << tile_shift;  // offset inside a sample's gradient
     const long long left = tn.seg_len - q.goff;
@@ -600,7 +703,7 @@ __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, i
 // One launch per element type DT and sample-group size RB (1..4): per-sample
 // operands and the single-sample remainder of shared operands run with RB = 1;
 // shared operands (weights) are read once per group of up to four samples.
-template <int DT, int FMASK, int RB>
+template <int DT, int FMASK, int RB, bool CAUSAL>
 __global__ void __launch_bounds__(kScoreThreads, kScoreCtasPerSm)
 score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
              int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
@@ -629,11 +732,11 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
     RingPos<RG::kStages> pos;  // both sides walk the ring in the same order
     int t = 0;        // tensor of the current tile; tiles only move forward
     if (producer) {
-        if (threadIdx.x == kConsumers) {
+        if (!CAUSAL && threadIdx.x == kConsumers) {  // causal tiles do not go through the ring
             for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
                 while (tile >= __ldg(tile_begin + t + 1)) ++t;
                 const Tensor& tn = tens[t];
-                const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
+                const TileGeom q = tile_geometry<RB, CAUSAL>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
                 constexpr int es = Elem<DT>::kBytes;
                 const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
                 const char* gb[RB];
@@ -679,7 +782,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
     for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         while (tile >= __ldg(tile_begin + t + 1)) ++t;
         const Tensor& tn = tens[t];
-        const TileGeom q = tile_geometry<RB>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
+        const TileGeom q = tile_geometry<RB, CAUSAL>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
         constexpr int es = Elem<DT>::kBytes;
         float2 inv2[2], nsc2[2];
 #pragma unroll
@@ -697,7 +800,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
             gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
             aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
         }
-        const int nchunks = aligned ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
+        const int nchunks = aligned && !CAUSAL ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
 
         double acc64[RB][NACC];
         Acc<NACC> acc[RB];
@@ -712,7 +815,9 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         flush_acc<NACC, RB>(acc, acc64);
         // what the ring did not carry
         const int done = (int)(((long long)nchunks * RG::kChunkBytes) / es);
-        if (done < q.n) {
+        if constexpr (CAUSAL) {
+            score_causal_rows<DT, FMASK>(vb, gb[0], q.n, q.goff >> tn.causal_shift, tn.causal_shift, inv2, nsc2, acc64);
+        } else if (done < q.n) {
             const char* gt[RB];
 #pragma unroll
             for (int r = 0; r < RB; ++r) gt[r] = gb[r] + (long long)done * es;
@@ -819,7 +924,7 @@ __global__ void job_prepare_kernel(SegmentJob* job, const void* values, const vo
     t.rgroups = 1;
     t.seg_base = 0;
     t.amax_preset = amax_preset;
-    t.pad = 0;
+    t.causal_shift = 0;
     job->tensor = t;
     job->tile_begin[0] = 0;
     job->tile_begin[1] = ntiles;
@@ -900,53 +1005,58 @@ int pick_tile_shift(long long scored_elems, int max_ctas) {
     return shift;
 }
 
-template <int DT, int FMASK, int RB>
+template <int DT, int FMASK, int RB, bool CAUSAL>
 static cudaError_t launch_score_inst(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                      int tile_shift, int max_ctas, const float* scales, double* partials,
                                      LaunchStatus* status, cudaStream_t st) {
     constexpr int smem = Ring<RB>::kSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB, CAUSAL>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(ntiles < (long long)max_ctas ? ntiles : (long long)max_ctas);
-    score_kernel<DT, FMASK, RB><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift, scales,
-                                                                   partials, status);
+    score_kernel<DT, FMASK, RB, CAUSAL><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift,
+                                                                           scales, partials, status);
     return cudaGetLastError();
 }
 
-template <int DT, int RB>
+template <int DT, int RB, bool CAUSAL>
 static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                    int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
                                    LaunchStatus* status, cudaStream_t st) {
     switch (fmask) {
-        case 1: return launch_score_inst<DT, 1, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 2: return launch_score_inst<DT, 2, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 3: return launch_score_inst<DT, 3, RB>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 1: return launch_score_inst<DT, 1, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 2: return launch_score_inst<DT, 2, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 3: return launch_score_inst<DT, 3, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
         default: return cudaErrorInvalidValue;
     }
 }
 
 template <int DT>
-static cudaError_t launch_score_dt(int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
-                                   int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                                   LaunchStatus* status, cudaStream_t st) {
+static cudaError_t launch_score_dt(int rb, int causal, const Tensor* tens, const long long* tile_begin, int T,
+                                   long long ntiles, int tile_shift, int max_ctas, int fmask, const float* scales,
+                                   double* partials, LaunchStatus* status, cudaStream_t st) {
+    if (causal) {  // causal operands are per-sample operands: one sample per read
+        if (rb != 1) return cudaErrorInvalidValue;
+        return launch_score_rb<DT, 1, true>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+    }
     switch (rb) {
-        case 1: return launch_score_rb<DT, 1>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 2: return launch_score_rb<DT, 2>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 3: return launch_score_rb<DT, 3>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 4: return launch_score_rb<DT, 4>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 1: return launch_score_rb<DT, 1, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 2: return launch_score_rb<DT, 2, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 3: return launch_score_rb<DT, 3, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 4: return launch_score_rb<DT, 4, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
         default: return cudaErrorInvalidValue;
     }
 }
 
 cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                          int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                         LaunchStatus* status, cudaStream_t st) {
+                         LaunchStatus* status, cudaStream_t st, int causal) {
     if (ntiles <= 0) return cudaSuccess;
     if (max_ctas < 1 || tile_shift < kMinTileShift || tile_shift > kMaxTileShift) return cudaErrorInvalidValue;
     if (dtype == 0)
-        return launch_score_dt<0>(rb, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        return launch_score_dt<0>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
     if (dtype == 1)
-        return launch_score_dt<1>(rb, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        return launch_score_dt<1>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
     return cudaErrorInvalidValue;
 }
 

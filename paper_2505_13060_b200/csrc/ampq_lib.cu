@@ -28,6 +28,7 @@ struct Operand {
     const void* grads = nullptr;
     long long numel = 0, grad_stride = 0;
     float amax_preset = -1.0f;
+    long long causal_T = 0;  // > 0: declared a stack of T x T lower-triangular matrices
     void* stage = nullptr;  // device staging for host-bound operands
     size_t stage_bytes = 0;
     int tensor = -1;        // index in the tables of the last score, or -1
@@ -185,6 +186,23 @@ bool layer_ready(const LayerRec& l) { return l.op[0].bound && l.op[1].bound; }
 
 long long extent_of(const LayerRec& l, const Operand& o) { return o.per_sample ? o.numel / l.R : o.numel; }
 
+// log2 T when the operand may be scored as a stack of lower-triangular T x T
+// matrices, else 0 (scored densely, which gives the same sums).  The triangular
+// path needs a power-of-two T in [64, 32768], whole matrices per sample, and
+// 16-byte aligned sample slices of values and gradients.
+int causal_shift_of(const LayerRec& l, const Operand& o, const Tensor& t) {
+    const long long T = o.causal_T;
+    if (T <= 0 || !o.per_sample || (T & (T - 1))) return 0;
+    int shift = 0;
+    while ((1LL << shift) < T) ++shift;
+    if (shift < kMinCausalShift || shift > kMaxCausalShift) return 0;
+    if (t.seg_len == 0 || t.seg_len % (T * T)) return 0;
+    const int es = o.dtype == AMPQ_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(t.values) & 15) || (reinterpret_cast<uintptr_t>(t.grads) & 15)) return 0;
+    if (l.R > 1 && (t.grad_stride * es) % 16) return 0;
+    return shift;
+}
+
 // Builds the host tables for every layer whose two operands are bound.
 int build_tables(ampq_ctx* ctx) {
     ctx->tens.clear(); ctx->amax_tile_begin.clear();
@@ -245,12 +263,15 @@ int build_tables(ampq_ctx* ctx) {
             t.partial_base = slots;
             t.seg_base = (int)ctx->segs.size();
             t.amax_preset = o.amax_preset;
+            t.causal_shift = causal_shift_of(l, o, t);
             // per-sample operands: one single-sample tile per (sample, value tile);
             // shared operands: value tiles x full groups of kMaxRB samples, plus one
             // remainder group of R mod kMaxRB samples
             long long my_tiles[kScoreClasses] = {};
             const int c0 = (o.dtype == AMPQ_F32 ? 0 : 1) * kMaxRB;  // classes of this operand's dtype
-            if (o.per_sample) {
+            if (t.causal_shift > 0) {
+                my_tiles[2 * kMaxRB + (o.dtype == AMPQ_F32 ? 0 : 1)] = (long long)l.R * t.tiles_per_seg;
+            } else if (o.per_sample) {
                 my_tiles[c0] = (long long)l.R * t.tiles_per_seg;
             } else {
                 my_tiles[c0 + kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
@@ -635,6 +656,16 @@ int ampq_get_amax(ampq_ctx* ctx, int layer_id, float* amax) {
     return AMPQ_OK;
 }
 
+int ampq_set_causal(ampq_ctx* ctx, int layer_id, int operand, long long T) {
+    int rc = check_layer(ctx, layer_id);
+    if (rc) return rc;
+    if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
+    if (T < 0) return fail(ctx, AMPQ_ERR_INVALID, "T must not be negative");
+    ctx->layers[layer_id].op[operand].causal_T = T;
+    ctx->dirty = true;
+    return AMPQ_OK;
+}
+
 int ampq_score(ampq_ctx* ctx) {
     if (!ctx) return AMPQ_ERR_INVALID;
     DeviceGuard g(ctx->device);
@@ -663,7 +694,10 @@ int ampq_score(ampq_ctx* ctx) {
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         for (int c = 0; c < kScoreClasses; ++c) {
             if (ctx->ntiles[c] <= 0) continue;
-            AMPQ_CUDA(launch_score(c / kMaxRB, c % kMaxRB + 1, ctx->d_tens.p, ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask, ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st), "score");
+            const bool causal = c >= 2 * kMaxRB;  // the last two classes: triangular operands, fp32 and bf16
+            AMPQ_CUDA(launch_score(causal ? c - 2 * kMaxRB : c / kMaxRB, causal ? 1 : c % kMaxRB + 1, ctx->d_tens.p,
+                                   ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask,
+                                   ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st, causal ? 1 : 0), "score");
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");

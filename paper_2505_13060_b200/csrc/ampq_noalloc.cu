@@ -73,7 +73,7 @@ __global__ void noalloc_prepare_kernel(NoAllocScratch* s, const void* values, co
     t.rgroups = 1;
     t.seg_base = 0;
     t.amax_preset = amax_preset;
-    t.pad = 0;
+    t.causal_shift = 0;
     s->tensor = t;
     s->tile_begin[0] = 0;
     s->tile_begin[1] = ntiles;
