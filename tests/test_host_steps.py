@@ -101,3 +101,28 @@ def test_baselines_match_oracle_and_never_beat_the_integer_program(ampq):
     ch = np.zeros(2, np.uint8)
     assert ampq.lib().ampq_select_in_order(2, o.ctypes.data, z.ctypes.data, z.ctypes.data, 1.0, ch.ctypes.data,
                                            None, None) == ampq.ERR_INVALID   # not a permutation
+
+
+def test_saved_layer_table_round_trips_bit_for_bit(ampq, tmp_path):
+    from paper_2505_13060_b200 import shard, table
+
+    rng = np.random.default_rng(14)
+    L, F = 23, 3
+    tab = np.concatenate([rng.uniform(0, 1, (L, 1)) ** 8, np.zeros((L, 1)), rng.uniform(0, 1e-3, (L, F - 1)),
+                          np.zeros((L, 1)), rng.uniform(0, 1e-3, (L, F - 1))], axis=1)
+    tab[3] = [5e-324, 0.0, 1.7976931348623157e308, 1e-300, 0.0, 0.1, 1.0 / 3.0]   # awkward doubles survive too
+    names = ["blk%d.fc" % i for i in range(L)]
+    path = str(tmp_path / "calib.json")
+    table.save_table(path, names, [0, 1, 2], tab, meta={"R": 8})
+    n2, f2, t2, meta = table.load_table(path)
+    assert n2 == names and f2 == [0, 1, 2] and meta == {"R": 8} and t2.tobytes() == tab.tobytes()
+    groups = [([i, i + 1], np.array([[0, 1, 2], [0, 1, 2]], np.uint8), np.array([0.0, 1.0 + i, 0.5 + i])) for i in range(0, 10, 2)]
+    tab[3] = tab[4]
+    table.save_table(path, names, [0, 1, 2], tab)
+    t3 = table.load_table(path)[2]
+    for mode in (ampq.D_MODEL, ampq.D_MEASURED):
+        a = shard.select_from_table(ampq, tab, F, groups, mode, 1e-3)
+        b = shard.select_from_table(ampq, t3, F, groups, mode, 1e-3)
+        assert a[0].tolist() == b[0].tolist() and a[1:] == b[1:]
+    with pytest.raises(ValueError):
+        table.save_table(path, names, [0, 1], tab)
