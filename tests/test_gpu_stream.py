@@ -183,3 +183,64 @@ def test_toy_mlp_hooks_and_predicted_vs_measured_loss_mse(ampq, orc):
     with torch.no_grad():
         assert [float(loss_of(r)) for r in range(3)] == g[:3]
     ctx.destroy()
+
+
+def test_algorithm_1_end_to_end_on_a_toy_model(ampq, orc):
+    """Algorithm 1 in one piece on a random MLP: partition the model graph,
+    calibrate through the hooks (sensitivities and mean-square loss), build the
+    MAC time-gain tables, solve the integer program for several thresholds tau.
+    The plan must equal the oracle's enumeration over the same tables, meet the
+    budget tau^2 E[g^2], and move from all-baseline (tau = 0) to all-FP8."""
+    from oracle import ampq_host_oracle as ho
+    from paper_2505_13060_b200 import hooks
+
+    torch.manual_seed(1)
+    R, tokens, width = 16, 32, 128
+    dims = [width, 256, 128, 256, 64, 10]
+    mods = []
+    for a, b in zip(dims[:-1], dims[1:]):
+        mods += [torch.nn.Linear(a, b), torch.nn.GELU()]
+    model = torch.nn.Sequential(*mods[:-1]).cuda()
+    xs = torch.randn(R, tokens, width, device="cuda")
+    ys = torch.randint(0, 10, (R, tokens), device="cuda")
+    # step 1: the graph is a chain Linear, GELU, Linear, ...; only the Linear vertices can be quantised
+    n = len(model)
+    edges = [(i, i + 1) for i in range(n - 1)]
+    quant = [isinstance(m, torch.nn.Linear) for m in model]
+    group_of, J = ampq.partition(n, edges, quant)
+    assert (group_of.tolist(), J) == ho.partition(n, edges, quant) and J == 5
+    # step 2: calibration
+    ctx = _ctx(ampq, (0, E4M3))
+    cal = hooks.Calibrator(ctx, model, R)
+    losses = []
+    cal.begin()
+    for r in range(R):
+        with cal.sample(r):
+            l = torch.nn.functional.cross_entropy(model(xs[r]), ys[r])
+            l.backward()
+            losses.append(float(l.detach()))
+    res = cal.end()
+    # step 3 stand-in: theoretical time gain from MAC counts (Sec. 2.3.2), one group per layer
+    lin = [m for m in model if isinstance(m, torch.nn.Linear)]
+    c_tabs, d_tabs = [], []
+    for j, (m, lid) in enumerate(zip(lin, cal.layer_ids)):
+        shape = (ampq.LINEAR, R * tokens, m.in_features, m.out_features)
+        c = ampq.gain_table(ampq.GAIN_MAC, [shape], [[0, 1]], [0.0, 1e-12])
+        assert c.tolist() == ho.gain_table(ho.GAIN_MAC, [shape], [[0, 1]], [0.0, 1e-12])
+        ctx.define_group([lid], np.array([[0, 1]], np.uint8), c)
+        c_tabs.append(c)
+        d_tabs.append(ctx.group_costs(j, ampq.D_MODEL))
+        assert d_tabs[-1][1] == res[j]["d_model"][1]
+    # step 4: the integer program under tau^2 E[g^2]
+    all_low = sum(d[1] for d in d_tabs)
+    plans = []
+    for tau in (0.0, 1e-4, 1e-3, 3e-3, 1e-2, 1.0):
+        budget = ampq.budget_from_tau(tau, losses)
+        assert budget == orc.budget_from_tau(tau, losses)
+        p, c, d = ctx.select(ampq.D_MODEL, budget)
+        want = orc.select_bruteforce(c_tabs, d_tabs, budget)
+        assert p.tolist() == want[0].tolist() and c == want[1] and d == want[2] and d <= budget
+        plans.append(int(p.sum()))
+    assert plans[0] == 0 and plans == sorted(plans)
+    assert plans[-1] == 5 or ampq.budget_from_tau(1.0, losses) < all_low
+    ctx.destroy()
