@@ -457,3 +457,51 @@ def test_operand_with_more_than_2_31_elements(ampq, orc):
     ctx.score()
     assert ctx.get_layer(lid)["amax"][0] == np.float32(100.0)
     ctx.destroy()
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_mix_of_layers_in_one_score(ampq, orc, seed):
+    """Forty layers of random element type, sample count, lengths (around tile
+    and chunk multiples) and alignments in ONE score, so that every scoring
+    launch walks tiles of many tensors, ring-fed and direct ones in turn."""
+    rng = np.random.default_rng(100 + seed)
+    g = torch.Generator(device="cuda").manual_seed(200 + seed)
+    ctx = _ctx(ampq, (0, E4M3, E5M2) if seed != 1 else (0, E5M2))
+    low = [E4M3, E5M2] if seed != 1 else [E5M2]
+    layers, keep = [], []
+
+    def length():
+        base = int(rng.choice([0, 1, 7, 2048, 4096, 32768, 65536, 3 * 32768, 1 << 19, (1 << 19) + 4096]))
+        return max(0, base + int(rng.choice([0, 0, 0, -1, 1, 8, -8, 5, 4095])))
+
+    for li in range(40):
+        dtype = torch.float32 if rng.random() < 0.3 else torch.bfloat16
+        es = 4 if dtype == torch.float32 else 2
+        R = int(rng.integers(1, 10))
+        nx, nw = length(), length()
+        offx, offw = (int(rng.integers(0, 8)) if rng.random() < 0.3 else 0 for _ in range(2))
+        stride = nw + (int(rng.integers(0, 9)) if rng.random() < 0.3 else 0)
+        bx = torch.empty(R * nx + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g)
+        bgx = torch.empty(R * nx + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g) * 1e-3
+        bw = torch.empty(nw + 16, dtype=dtype, device="cuda").normal_(0, 0.02, generator=g)
+        bgw = torch.empty(R * stride + 16, dtype=dtype, device="cuda").normal_(0, 1, generator=g) * 1e-3
+        keep += [bx, bgx, bw, bgw]
+        lid = ctx.register_layer(ampq.LINEAR, "mix%d" % li, R)
+        code = ampq.torch_dtype_code(bx)
+        ctx.bind_operand(lid, 0, code, bx.data_ptr() + offx * es, R * nx, True, bgx.data_ptr() + offx * es, nx)
+        ctx.bind_operand(lid, 1, code, bw.data_ptr() + offw * es, nw, False, bgw.data_ptr() + offw * es, stride)
+
+        class LT:
+            pass
+
+        lt = LT()
+        lt.spec = synth.LayerSpec("mix%d" % li, synth.LINEAR, R, dtype, synth.OperandSpec((R, nx), True),
+                                  synth.OperandSpec((nw,), False))
+        lt.values = [bx[offx:offx + R * nx].reshape(R, nx), bw[offw:offw + nw]]
+        lt.grads = [bgx[offx:offx + R * nx].reshape(R, nx),
+                    torch.stack([bgw[offw + r * stride: offw + r * stride + nw] for r in range(R)])]
+        layers.append((lid, lt))
+    ctx.score()
+    for lid, lt in layers:
+        compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, low, threads=8), 1 + len(low), lt.spec.name)
+    ctx.destroy()
