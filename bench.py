@@ -447,6 +447,10 @@ def run_b200(args):
             "roofline": roofline, "cpu_baseline": cpu,
             "check": check,
             "pct_of_hbm_peak": {"measured_%.0f" % peak: 100.0 * value / peak, "datasheet_8000": 100.0 * value / 8000.0},
+            # every byte the step reads (the amax pass reads each operand once more), all ranks
+            "whole_pass_traffic": {"algorithmic_bytes_per_gpu": scored_bytes + value_bytes,
+                                   "gbs": world * (scored_bytes + value_bytes) / (ms_per_step * 1e-3) / 1e9,
+                                   "frac_of_measured_peak": (scored_bytes + value_bytes) / (ms_per_step * 1e-3) / 1e9 / peak},
         }
         print(json.dumps(line), flush=True)
     if dist is not None:
