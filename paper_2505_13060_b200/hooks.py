@@ -1,8 +1,10 @@
 """Calibration of a PyTorch model through module hooks (Algorithm 1 step 2:
 "wrap the model", then one high-precision forward and backward per sample).
 
-``Calibrator`` registers every ``torch.nn.Linear`` of a model as a layer of a
-scoring context.  While a sample runs, a forward hook keeps the layer input X
+``Calibrator`` registers every ``torch.nn.Linear`` of a model as a linear layer
+of a scoring context and every ``BatchedMatmul`` (a module that only wraps
+``torch.matmul``, so that the attention products Q K^T and P V are visible to
+hooks) as a batched GEMM with operands X0, X1 (Sec. 2.2).  While a sample runs, a forward hook keeps the layer input X
 and a backward hook receives dL/dX and dL/dY; the sample's weight gradient
 dL/dW = dL/dY^T X is formed by a torch matmul (the GEMM that produces a gradient
 is not part of the scoring path) and both operands of the layer are streamed to
@@ -23,6 +25,14 @@ import torch
 from . import binding as ampq
 
 
+class BatchedMatmul(torch.nn.Module):
+    """``torch.matmul(a, b)`` as a module: a batched GEMM layer Y = X0 (x) X1 whose
+    two operands and their gradients the calibrator can see."""
+
+    def forward(self, a, b):
+        return torch.matmul(a, b)
+
+
 class Calibrator:
     def __init__(self, ctx: "ampq.Context", model: torch.nn.Module, R: int):
         self.ctx, self.model, self.R = ctx, model, R
@@ -31,6 +41,9 @@ class Calibrator:
             if isinstance(m, torch.nn.Linear):
                 self.modules.append((name, m))
                 self.layer_ids.append(ctx.register_layer(ampq.LINEAR, name, R))
+            elif isinstance(m, BatchedMatmul):
+                self.modules.append((name, m))
+                self.layer_ids.append(ctx.register_layer(ampq.BGEMM, name, R))
         self._r = None
         self._x = {}
         self._keep = []   # tensors borrowed by the library until the stream has caught up
@@ -40,12 +53,20 @@ class Calibrator:
     def _fwd(self, idx):
         def hook(module, inputs, output):
             if self._r is not None:
-                self._x[idx] = inputs[0].detach()
+                self._x[idx] = tuple(t.detach() for t in inputs) if isinstance(module, BatchedMatmul) else inputs[0].detach()
         return hook
 
     def _bwd(self, idx):
         def hook(module, grad_input, grad_output):
             if self._r is None:
+                return
+            if isinstance(module, BatchedMatmul):   # both operands belong to the sample
+                lid = self.layer_ids[idx]
+                for k, (x, gx) in enumerate(zip(self._x.pop(idx), grad_input)):
+                    x = x.contiguous()
+                    gx = (torch.zeros_like(x) if gx is None else gx.detach().reshape(x.shape)).contiguous()
+                    self.ctx.stream_sample(lid, k, self._r, ampq.torch_dtype_code(x), x.data_ptr(), gx.data_ptr(), x.numel())
+                    self._keep += [x, gx]
                 return
             x = self._x.pop(idx).contiguous()
             gy = grad_output[0].detach()
@@ -99,6 +120,20 @@ class Calibrator:
         for idx, (_, m) in enumerate(self.modules):
             fmt = fmt_of_layer[idx]
             if not fmt:
+                continue
+            if isinstance(m, BatchedMatmul):   # both inputs rounded, each with its own measured amax
+
+                def pre2(module, inputs, fmt=fmt):
+                    outs = []
+                    for x in inputs:
+                        x = x.contiguous()
+                        out = torch.empty_like(x)
+                        self.ctx.fake_quant(ampq.torch_dtype_code(x), fmt, x.data_ptr(), x.numel(), -1.0, out.data_ptr())
+                        self._keep.append(x)
+                        outs.append(out)
+                    return tuple(outs)
+
+                handles.append(m.register_forward_pre_hook(pre2))
                 continue
             w = m.weight.data
             saved.append((m, w.clone()))

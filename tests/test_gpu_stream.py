@@ -244,3 +244,90 @@ def test_algorithm_1_end_to_end_on_a_toy_model(ampq, orc):
     assert plans[0] == 0 and plans == sorted(plans)
     assert plans[-1] == 5 or ampq.budget_from_tau(1.0, losses) < all_low
     ctx.destroy()
+
+
+class _Attention(torch.nn.Module):
+    """One causal self-attention block with its two batched products as modules."""
+
+    def __init__(self, width, heads):
+        super().__init__()
+        from paper_2505_13060_b200 import hooks
+
+        self.h, self.d = heads, width // heads
+        self.q, self.k, self.v, self.o = (torch.nn.Linear(width, width) for _ in range(4))
+        self.qk, self.av = hooks.BatchedMatmul(), hooks.BatchedMatmul()
+        self.head = torch.nn.Linear(width, 8)
+
+    def forward(self, x):   # x: [tokens, width]
+        T = x.shape[0]
+        split = lambda t: t.reshape(T, self.h, self.d).transpose(0, 1)   # [heads, tokens, d]
+        s = self.qk(split(self.q(x)), split(self.k(x)).transpose(1, 2)) / self.d ** 0.5
+        mask = torch.ones(T, T, dtype=torch.bool, device=x.device).triu(1)
+        p = torch.softmax(s.masked_fill(mask, float("-inf")), dim=-1)
+        y = self.av(p, split(self.v(x))).transpose(0, 1).reshape(T, -1)
+        return self.head(x + self.o(y))
+
+
+def test_attention_block_with_batched_products_through_hooks(ampq, orc):
+    """Linear and batched-GEMM layers of a causal attention block calibrated
+    through the hooks: the two products against the oracle from tensors captured
+    independently, and predicted against measured loss MSE with all seven
+    layers (five of them the paper's attention sub-graph) in E4M3."""
+    from paper_2505_13060_b200 import hooks
+
+    torch.manual_seed(3)
+    R, tokens, width, heads = 32, 64, 128, 2
+    model = _Attention(width, heads).cuda()
+    xs = torch.randn(R, tokens, width, device="cuda")
+    ys = torch.randint(0, 8, (R, tokens), device="cuda")
+    loss_of = lambda r: torch.nn.functional.cross_entropy(model(xs[r]), ys[r])
+    ctx = _ctx(ampq, (0, E4M3))
+    cal = hooks.Calibrator(ctx, model, R)
+    names = [n for n, _ in cal.modules]
+    assert sorted(names) == sorted(["q", "k", "v", "o", "qk", "av", "head"])
+    cap = {"qk": [], "av": []}
+    hs = []
+    for key in cap:
+        m = getattr(model, key)
+        hs.append(m.register_forward_hook(lambda mod, i, o, key=key: cap[key].append([t.detach().clone() for t in i])))
+        hs.append(m.register_full_backward_hook(lambda mod, gi, go, key=key: cap[key][-1].extend(t.detach().clone() for t in gi)))
+    g = []
+    cal.begin()
+    for r in range(R):
+        with cal.sample(r):
+            l = loss_of(r)
+            l.backward()
+            g.append(float(l.detach()))
+    res = cal.end()
+    for h in hs:
+        h.remove()
+    for key in ("qk", "av"):
+        a = torch.stack([c[0].contiguous() for c in cap[key]])
+        b = torch.stack([c[1].contiguous() for c in cap[key]])
+        ga = torch.stack([c[2].contiguous() for c in cap[key]])
+        gb = torch.stack([c[3].contiguous() for c in cap[key]])
+
+        class LT:
+            pass
+
+        lt = LT()
+        lt.spec = synth.LayerSpec(key, synth.BGEMM, R, torch.float32, synth.OperandSpec(tuple(a.shape), True),
+                                  synth.OperandSpec(tuple(b.shape), True))
+        lt.values, lt.grads = [a, b], [ga, gb]
+        # without presets every sample was scaled by its own amax: compare sample by sample
+        lid = cal.layer_ids[names.index(key)]
+        for k, (v, gr) in enumerate(((a, ga), (b, gb))):
+            got = ctx.get_operand(lid, k)
+            for r in (0, R // 2, R - 1):
+                hv, hg = synth.to_numpy(v[r]), synth.to_numpy(gr[r])
+                _, _, _, seg = orc.score_operand(hv.reshape(-1), hg.reshape(1, -1), 1, False, [E4M3])
+                assert_close(got[r], seg[0], "%s operand %d sample %d" % (key, k, r))
+        if key == "av":
+            assert float(a[0, 0].triu(1).abs().max()) == 0.0   # P is causal: exact zeros above the diagonal
+    # predicted against measured with everything in E4M3 (per-call scales on both sides)
+    d_meas = sum(r_["d_meas"][1] for r_ in res)
+    with torch.no_grad(), cal.quantised([E4M3] * len(names)):
+        gq = [float(loss_of(r)) for r in range(R)]
+    measured = float(np.mean((np.array(gq) - np.array(g)) ** 2))
+    assert 0.4 < measured / d_meas < 2.5, (measured, d_meas)
+    ctx.destroy()
