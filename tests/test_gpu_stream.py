@@ -177,6 +177,7 @@ def test_toy_mlp_hooks_and_predicted_vs_measured_loss_mse(ampq, orc):
         gq = [float(loss_of(r)) for r in range(R)]
     measured = float(np.mean((np.array(gq) - np.array(g)) ** 2))
     assert measured > 0
+    print("toy MLP: measured / predicted loss MSE = %.3f (measured error), %.3f (noise model)" % (measured / d_meas, measured / d_model))
     assert 0.5 < measured / d_meas < 2.0, (measured, d_meas, d_model)
     assert 0.15 < measured / d_model < 1.2, (measured, d_meas, d_model)
     # nothing is left quantised
@@ -329,5 +330,6 @@ def test_attention_block_with_batched_products_through_hooks(ampq, orc):
     with torch.no_grad(), cal.quantised([E4M3] * len(names)):
         gq = [float(loss_of(r)) for r in range(R)]
     measured = float(np.mean((np.array(gq) - np.array(g)) ** 2))
+    print("attention block: measured / predicted loss MSE = %.3f" % (measured / d_meas))
     assert 0.4 < measured / d_meas < 2.5, (measured, d_meas)
     ctx.destroy()
