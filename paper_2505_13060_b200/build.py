@@ -35,15 +35,19 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, out: str | None = None, defines=()) -> str:
+    """Builds the library.  ``out``/``defines`` make a second build beside the
+    default one, e.g. ``defines=["AMPQ_BOUNDS_CHECK"]`` for the self-checking
+    debug build (load it with the AMPQ_LIBRARY environment variable)."""
+    lib = out or LIB
+    if out is None and not force and not needs_build():
         return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-shared", "-o", tmp]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
+    tmp = lib + ".tmp.%d" % os.getpid()
+    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-D" + d for d in defines]
+    cmd += ["-shared", "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

@@ -91,6 +91,7 @@ struct SegmentJob {
 struct LaunchStatus {
     int nonfinite;  // set when some tensor's amax is Inf/NaN
     int timeout;    // set when a wait inside the scoring kernel ran out
+    int bounds;     // set by a -DAMPQ_BOUNDS_CHECK build when a tile falls outside its tensor
 };
 
 }  // namespace ampq

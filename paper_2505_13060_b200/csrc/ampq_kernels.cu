@@ -130,6 +130,7 @@ __global__ void init_amax_kernel(const Tensor* __restrict__ tens, int T,
     if (t == 0) {
         status->nonfinite = 0;
         status->timeout = 0;
+        status->bounds = 0;
     }
     if (t < T) {
         float p = tens[t].amax_preset;
@@ -147,6 +148,9 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
     const Tensor& tn = tens[t];
     const long long first = (tile - __ldg(tile_begin + t)) * (long long)kAmaxTileElems;
     const long long left = tn.numel - first;
+#ifdef AMPQ_BOUNDS_CHECK
+    if (first < 0 || left <= 0) return;  // a tile outside its tensor is not read (the scoring pass reports it)
+#endif
     const int n = left < kAmaxTileElems ? (int)left : kAmaxTileElems;
     const int es = tn.dtype == 0 ? 4 : 2;
     const char* base = reinterpret_cast<const char*>(tn.values) + first * es;
@@ -689,6 +693,23 @@ __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, i
     return q;
 }
 
+// Debug builds (-DAMPQ_BOUNDS_CHECK): a tile whose element range, samples or
+// partial slots fall outside what its tensor owns is reported in the status
+// word and skipped by the producer and the scoring warps alike, instead of
+// being read.  The check costs a few compares per tile and is compiled out of
+// release builds.
+template <int RB>
+__device__ __forceinline__ bool tile_in_bounds(const Tensor& tn, const TileGeom& q) {
+#ifdef AMPQ_BOUNDS_CHECK
+    const long long vals = tn.per_sample ? tn.numel : tn.seg_len;
+    return q.n > 0 && q.goff >= 0 && q.goff + q.n <= tn.seg_len && q.voff >= 0 && q.voff + q.n <= vals &&
+           q.r0 >= 0 && q.r0 + RB <= tn.R && q.slot0 >= tn.partial_base &&
+           q.slot0 + (long long)(RB - 1) * tn.tiles_per_seg < tn.partial_base + (long long)tn.R * tn.tiles_per_seg;
+#else
+    return true;
+#endif
+}
+
 // The scoring kernel.  Persistent: CTA b takes tiles b, b + gridDim.x, ... of
 // the launch's tile table.  Warps 0..7 score; warp 8 is the producer: one lane
 // streams every full 16-byte-aligned chunk of the value tile and of its RB
@@ -746,7 +767,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
                     gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
                     aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
                 }
-                const int nchunks = aligned ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
+                const int nchunks = aligned && tile_in_bounds<RB>(tn, q) ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
                 for (int c = 0; c < nchunks; ++c) {
                     // the stage must have been handed back once per earlier lap
                     if (it >= (unsigned)RG::kStages && !mbar_wait(empty + pos.stage, pos.parity ^ 1u, s_abort)) break;
@@ -799,6 +820,11 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         for (int r = 0; r < RB; ++r) {
             gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
             aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
+        }
+        const bool inside = tile_in_bounds<RB>(tn, q);
+        if (!inside) {  // only in a bounds-checking build: report, score nothing, move on
+            if (threadIdx.x == 0) atomicExch(&status->bounds, 1);
+            continue;
         }
         const int nchunks = aligned && !CAUSAL ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
 

@@ -380,6 +380,8 @@ int sync_results(ampq_ctx* ctx) {
         AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
         ctx->pending = false;
     }
+    if (!ctx->tens.empty() && ctx->h_status.p->bounds)
+        return fail(ctx, AMPQ_ERR_CUDA, "bounds check: a scoring tile fell outside its tensor (library bug); the results of this score are invalid");
     if (!ctx->tens.empty() && ctx->h_status.p->timeout)
         return fail(ctx, AMPQ_ERR_TIMEOUT, "a bounded wait inside the scoring kernel ran out; the results of this score are invalid");
     return AMPQ_OK;
