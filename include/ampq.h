@@ -59,7 +59,7 @@ enum {
     AMPQ_ERR_CUDA = -4,        /* a CUDA call failed; see ampq_last_error           */
     AMPQ_ERR_NONFINITE = -5,   /* a scored operand holds Inf or NaN                 */
     AMPQ_ERR_INFEASIBLE = -6,  /* no assignment meets the budget                    */
-    AMPQ_ERR_TOO_LARGE = -7,   /* selection exceeded its state limit                */
+    AMPQ_ERR_TOO_LARGE = -7,   /* too large: selection state limit, tile count, fixed scratch */
     AMPQ_ERR_NOMEM = -8,
     AMPQ_ERR_TIMEOUT = -9      /* a bounded wait inside a kernel ran out; results invalid */
 };
