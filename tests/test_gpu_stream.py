@@ -211,9 +211,20 @@ def test_algorithm_1_end_to_end_on_a_toy_model(ampq, orc):
     quant = [isinstance(m, torch.nn.Linear) for m in model]
     group_of, J = ampq.partition(n, edges, quant)
     assert (group_of.tolist(), J) == ho.partition(n, edges, quant) and J == 5
-    # step 2: calibration
+    # step 2: calibration (with every layer's tensors captured on the side for the oracle)
     ctx = _ctx(ampq, (0, E4M3))
     cal = hooks.Calibrator(ctx, model, R)
+    lin = [m for m in model if isinstance(m, torch.nn.Linear)]
+    cap = [dict(x=[], gx=[], gy=[]) for _ in lin]
+    hs = []
+    for c_, m in zip(cap, lin):
+        hs.append(m.register_forward_hook(lambda mod, i, o, c_=c_: c_["x"].append(i[0].detach().clone())))
+
+        def grab(mod, gi, go, c_=c_):
+            c_["gx"].append(None if gi[0] is None else gi[0].detach().clone())
+            c_["gy"].append(go[0].detach().clone())
+
+        hs.append(m.register_full_backward_hook(grab))
     losses = []
     cal.begin()
     for r in range(R):
@@ -222,26 +233,41 @@ def test_algorithm_1_end_to_end_on_a_toy_model(ampq, orc):
             l.backward()
             losses.append(float(l.detach()))
     res = cal.end()
+    for h in hs:
+        h.remove()
+    # the oracle's sensitivities from the captured tensors: s^r = S(X, dX) + S(W, dW), s = mean_r
+    s_oracle = []
+    for c_, m in zip(cap, lin):
+        w = m.weight.detach()
+        tot = 0.0
+        for r in range(R):
+            x, gy = c_["x"][r], c_["gy"][r]
+            gx = c_["gx"][r] if c_["gx"][r] is not None else gy @ w
+            gw = gy.t() @ x
+            for v, gr in ((x, gx), (w, gw)):
+                tot += orc.score_segment(synth.to_numpy(v), synth.to_numpy(gr.contiguous()), [E4M3], [1.0], [1.0])[0]
+        s_oracle.append(tot / R)
     # step 3 stand-in: theoretical time gain from MAC counts (Sec. 2.3.2), one group per layer
-    lin = [m for m in model if isinstance(m, torch.nn.Linear)]
-    c_tabs, d_tabs = [], []
+    c_orc, d_gpu, d_orc = [], [], []
     for j, (m, lid) in enumerate(zip(lin, cal.layer_ids)):
         shape = (ampq.LINEAR, R * tokens, m.in_features, m.out_features)
         c = ampq.gain_table(ampq.GAIN_MAC, [shape], [[0, 1]], [0.0, 1e-12])
-        assert c.tolist() == ho.gain_table(ho.GAIN_MAC, [shape], [[0, 1]], [0.0, 1e-12])
+        c_orc.append(ho.gain_table(ho.GAIN_MAC, [shape], [[0, 1]], [0.0, 1e-12]))
+        assert c.tolist() == c_orc[-1]
         ctx.define_group([lid], np.array([[0, 1]], np.uint8), c)
-        c_tabs.append(c)
-        d_tabs.append(ctx.group_costs(j, ampq.D_MODEL))
-        assert d_tabs[-1][1] == res[j]["d_model"][1]
-    # step 4: the integer program under tau^2 E[g^2]
-    all_low = sum(d[1] for d in d_tabs)
+        d_gpu.append(ctx.group_costs(j, ampq.D_MODEL))
+        d_orc.append(np.array([0.0, orc.alpha(3) * s_oracle[j]]))
+        assert_close(d_gpu[-1][1], d_orc[-1][1], "d_model of layer %d" % j)
+    # step 4: the integer program under tau^2 E[g^2]: the library on its tables, the oracle on its own
+    all_low = sum(d[1] for d in d_orc)
     plans = []
     for tau in (0.0, 1e-4, 1e-3, 3e-3, 1e-2, 1.0):
         budget = ampq.budget_from_tau(tau, losses)
         assert budget == orc.budget_from_tau(tau, losses)
         p, c, d = ctx.select(ampq.D_MODEL, budget)
-        want = orc.select_bruteforce(c_tabs, d_tabs, budget)
-        assert p.tolist() == want[0].tolist() and c == want[1] and d == want[2] and d <= budget
+        want = orc.select_bruteforce(c_orc, d_orc, budget)
+        assert p.tolist() == want[0].tolist() and c == want[1] and d <= budget
+        assert_close(d, want[2], "selected loss MSE") if want[2] else None
         plans.append(int(p.sum()))
     assert plans[0] == 0 and plans == sorted(plans)
     assert plans[-1] == 5 or ampq.budget_from_tau(1.0, losses) < all_low
