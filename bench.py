@@ -62,6 +62,8 @@ def parse_args():
     ap.add_argument("--workload", default="llama70b", choices=["llama70b", "llama7b", "attention"],
                     help="llama70b is the benchmark; llama7b (3.2 GB per block) and attention (the two BGEMMs of one "
                          "attention layer per block, 2.55 GB) are side measurements, never the headline")
+    ap.add_argument("--model-only", action="store_true",
+                    help="side measurement: score only the paper's model term S (no amax pass, no FP8 cast)")
     ap.add_argument("--causal", action="store_true",
                     help="attention workload: declare the softmax operand causal so that its zero triangle is not read")
     ap.add_argument("--layers", default="",
@@ -316,6 +318,8 @@ def run_b200(args):
     stream = torch.cuda.Stream(device=dev)
     ctx = ampq.Context(local_rank, stream.cuda_stream)
     ctx.set_formats(fmts)
+    if args.model_only:
+        ctx.set_measured(False)
     slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev, seed=100 + rank, causal=args.causal)
     value_bytes = args.blocks * sum(sp.value_bytes() for sp in specs)
     ctx.set_timing(True)
@@ -436,7 +440,7 @@ def run_b200(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else "") + ("[causal]" if args.causal else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
+                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else "") + ("[causal]" if args.causal else "") + ("[model term only]" if args.model_only else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
                 "tokens_per_sample": specs[0].op0.shape[-2], "operand_dtype": "bf16", "formats": args.formats,
                 "scored_bytes_per_step_per_gpu": scored_bytes, "resident_blocks": nres,
                 "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block" % (nres, block_gb),

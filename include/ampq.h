@@ -134,6 +134,15 @@ int ampq_set_causal(ampq_ctx *ctx, int layer_id, int operand, long long T);
 enum { AMPQ_SCALE_AMAX = 0, AMPQ_SCALE_POW2 = 1 };
 int ampq_set_scale_mode(ampq_ctx *ctx, int mode);
 
+/* on = 0: score only the paper's own term, S = sum (z g)^2, from which
+ * d_model_f = alpha_f s follows (Sec. 2.2); the amax pass, the scales and the FP8
+ * cast are skipped, every measured value (D_f, d_meas) reads 0, amax reads 0
+ * (or the preset) and the scales are those of that amax.  One read of operand and
+ * gradient instead of two of the operand.  Inf/NaN in an operand is then not
+ * detected up front: it shows as a non-finite S.  on = 1 (default): both terms.
+ * Applies to ampq_score and ampq_stream_sample. */
+int ampq_set_measured(ampq_ctx *ctx, int on);
+
 /* Only the first step of ampq_score: amax of every bound operand of every fully
  * bound layer (preset ones keep their preset), asynchronously on the stream.
  * ampq_get_amax (synchronises) then gives amax[2] of a layer; it also works

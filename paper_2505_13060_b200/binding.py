@@ -37,7 +37,7 @@ EXPORTS = [
     "ampq_all_lowp_cost", "ampq_select", "ampq_select_tables", "ampq_score_segment_noalloc",
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
-    "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal",
+    "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal", "ampq_set_measured",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -87,6 +87,7 @@ def lib():
     L.ampq_stream_end.argtypes = [vp]
     L.ampq_fake_quant.argtypes = [vp, i, i, vp, ll, C.c_float, vp]
     L.ampq_set_causal.argtypes = [vp, i, i, ll]
+    L.ampq_set_measured.argtypes = [vp, i]
     L.ampq_set_scale_mode.argtypes = [vp, i]
     L.ampq_measure_amax.argtypes = [vp]
     L.ampq_get_amax.argtypes = [vp, i, vp]
@@ -264,6 +265,9 @@ class Context:
 
     def set_causal(self, layer_id: int, operand: int, T: int):
         self._check(lib().ampq_set_causal(self._h, layer_id, operand, T))
+
+    def set_measured(self, on: bool):
+        self._check(lib().ampq_set_measured(self._h, 1 if on else 0))
 
     def set_scale_mode(self, mode: int):
         self._check(lib().ampq_set_scale_mode(self._h, mode))

@@ -297,7 +297,7 @@ template <int FMASK>
 struct Fm {
     static constexpr int kLow = (FMASK & 1) + ((FMASK >> 1) & 1);
     static constexpr int kAcc = 1 + kLow;
-    static constexpr int kFmt0 = (FMASK & 1) ? kMaskE4M3 : kMaskE5M2;
+    static constexpr int kFmt0 = (FMASK & 1) ? kMaskE4M3 : kMaskE5M2;  // unused when FMASK = 0 (S only)
     static constexpr int kFmt1 = kMaskE5M2;
 };
 
@@ -313,15 +313,17 @@ __device__ __forceinline__ void accumulate_pairs(const float2 (&z)[NP], const fl
                                                  Acc<Fm<FMASK>::kAcc> (&acc)[RB]) {
 #pragma unroll
     for (int k = 0; k < NP; ++k) {
-        float2 ne0 = neg_err_pair<Fm<FMASK>::kFmt0>(z[k], inv2[0], nsc2[0]);
-        float2 ne1;
+        float2 ne0, ne1;
+        if constexpr (Fm<FMASK>::kLow >= 1) ne0 = neg_err_pair<Fm<FMASK>::kFmt0>(z[k], inv2[0], nsc2[0]);
         if constexpr (Fm<FMASK>::kLow == 2) ne1 = neg_err_pair<Fm<FMASK>::kFmt1>(z[k], inv2[1], nsc2[1]);
 #pragma unroll
         for (int r = 0; r < RB; ++r) {
             float2 p = __fmul2_rn(z[k], g[r][k]);
             acc[r].v[0] = __ffma2_rn(p, p, acc[r].v[0]);
-            float2 t0 = __fmul2_rn(ne0, g[r][k]);
-            acc[r].v[1] = __ffma2_rn(t0, t0, acc[r].v[1]);
+            if constexpr (Fm<FMASK>::kLow >= 1) {
+                float2 t0 = __fmul2_rn(ne0, g[r][k]);
+                acc[r].v[1] = __ffma2_rn(t0, t0, acc[r].v[1]);
+            }
             if constexpr (Fm<FMASK>::kLow == 2) {
                 float2 t1 = __fmul2_rn(ne1, g[r][k]);
                 acc[r].v[Fm<FMASK>::kAcc - 1] = __ffma2_rn(t1, t1, acc[r].v[Fm<FMASK>::kAcc - 1]);
@@ -464,7 +466,7 @@ struct RingPos {
 template <int NACC, int RB>
 __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], double* s_red,
                                                  double* __restrict__ partials, long long slot0,
-                                                 long long slot_stride) {
+                                                 long long slot_stride, int out_stride) {
     constexpr int NV = RB * NACC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -483,7 +485,7 @@ __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], 
 #pragma unroll
         for (int w = 0; w < kConsumers / 32; ++w) x += s_red[w * NV + threadIdx.x];
         const int r = threadIdx.x / NACC, a = threadIdx.x % NACC;
-        partials[(slot0 + r * slot_stride) * NACC + a] = x;
+        partials[(slot0 + r * slot_stride) * out_stride + a] = x;  // out_stride >= NACC doubles per slot
     }
 }
 
@@ -728,7 +730,7 @@ template <int DT, int FMASK, int RB, bool CAUSAL>
 __global__ void __launch_bounds__(kScoreThreads, kScoreCtasPerSm)
 score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
              int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
-             LaunchStatus* __restrict__ status) {
+             LaunchStatus* __restrict__ status, int out_stride) {
     using RG = Ring<RB>;
     constexpr int NACC = Fm<FMASK>::kAcc;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -850,7 +852,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
             score_direct<DT, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
         }
         reduce_and_store<NACC, RB>(acc64, s_red + red_block * (kConsumers / 32) * RB * NACC, partials, q.slot0,
-                                   tn.tiles_per_seg);
+                                   tn.tiles_per_seg, out_stride);
         red_block ^= 1;
     }
 }
@@ -1034,25 +1036,27 @@ int pick_tile_shift(long long scored_elems, int max_ctas) {
 template <int DT, int FMASK, int RB, bool CAUSAL>
 static cudaError_t launch_score_inst(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                      int tile_shift, int max_ctas, const float* scales, double* partials,
-                                     LaunchStatus* status, cudaStream_t st) {
+                                     LaunchStatus* status, cudaStream_t st, int out_stride) {
     constexpr int smem = Ring<RB>::kSmemBytes;
+    if (out_stride < Fm<FMASK>::kAcc) out_stride = Fm<FMASK>::kAcc;
     cudaError_t e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB, CAUSAL>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(ntiles < (long long)max_ctas ? ntiles : (long long)max_ctas);
     score_kernel<DT, FMASK, RB, CAUSAL><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift,
-                                                                           scales, partials, status);
+                                                                           scales, partials, status, out_stride);
     return cudaGetLastError();
 }
 
 template <int DT, int RB, bool CAUSAL>
 static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                                    int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                                   LaunchStatus* status, cudaStream_t st) {
+                                   LaunchStatus* status, cudaStream_t st, int out_stride) {
     switch (fmask) {
-        case 1: return launch_score_inst<DT, 1, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 2: return launch_score_inst<DT, 2, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
-        case 3: return launch_score_inst<DT, 3, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st);
+        case 0: return launch_score_inst<DT, 0, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st, out_stride);
+        case 1: return launch_score_inst<DT, 1, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st, out_stride);
+        case 2: return launch_score_inst<DT, 2, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st, out_stride);
+        case 3: return launch_score_inst<DT, 3, RB, CAUSAL>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, scales, partials, status, st, out_stride);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -1060,29 +1064,29 @@ static cudaError_t launch_score_rb(const Tensor* tens, const long long* tile_beg
 template <int DT>
 static cudaError_t launch_score_dt(int rb, int causal, const Tensor* tens, const long long* tile_begin, int T,
                                    long long ntiles, int tile_shift, int max_ctas, int fmask, const float* scales,
-                                   double* partials, LaunchStatus* status, cudaStream_t st) {
+                                   double* partials, LaunchStatus* status, cudaStream_t st, int out_stride) {
     if (causal) {  // causal operands are per-sample operands: one sample per read
         if (rb != 1) return cudaErrorInvalidValue;
-        return launch_score_rb<DT, 1, true>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        return launch_score_rb<DT, 1, true>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
     }
     switch (rb) {
-        case 1: return launch_score_rb<DT, 1, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 2: return launch_score_rb<DT, 2, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 3: return launch_score_rb<DT, 3, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
-        case 4: return launch_score_rb<DT, 4, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        case 1: return launch_score_rb<DT, 1, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
+        case 2: return launch_score_rb<DT, 2, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
+        case 3: return launch_score_rb<DT, 3, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
+        case 4: return launch_score_rb<DT, 4, false>(tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
         default: return cudaErrorInvalidValue;
     }
 }
 
 cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                          int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                         LaunchStatus* status, cudaStream_t st, int causal) {
+                         LaunchStatus* status, cudaStream_t st, int causal, int out_stride) {
     if (ntiles <= 0) return cudaSuccess;
     if (max_ctas < 1 || tile_shift < kMinTileShift || tile_shift > kMaxTileShift) return cudaErrorInvalidValue;
     if (dtype == 0)
-        return launch_score_dt<0>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        return launch_score_dt<0>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
     if (dtype == 1)
-        return launch_score_dt<1>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st);
+        return launch_score_dt<1>(rb, causal, tens, tile_begin, T, ntiles, tile_shift, max_ctas, fmask, scales, partials, status, st, out_stride);
     return cudaErrorInvalidValue;
 }
 

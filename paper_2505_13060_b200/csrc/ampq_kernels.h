@@ -23,12 +23,14 @@ cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* sc
                           LaunchStatus* status, cudaStream_t st, int pow2 = 0);
 // One launch per element type (0 = fp32, 1 = bf16) and sample-group size rb =
 // 1..kMaxRB, each with its own tile table; causal = 1 (rb = 1 only): the
-// table holds triangular operands (Tensor::causal_shift > 0).
+// table holds triangular operands (Tensor::causal_shift > 0).  fmask = 0 scores
+// only S (no cast, scales unused).  out_stride = doubles per partial slot when
+// that is more than the kernel's own accumulator count (0: exactly that count).
 // Tiles hold 2^tile_shift elements; the persistent grid has at most max_ctas CTAs
 // (two per SM is the intended residency).
 cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                          int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
-                         LaunchStatus* status, cudaStream_t st, int causal = 0);
+                         LaunchStatus* status, cudaStream_t st, int causal = 0, int out_stride = 0);
 // Largest tile shift in [kMinTileShift, kMaxTileShift] that still gives a grid of
 // max_ctas CTAs a few dozen tiles each (or the smallest shift when even that does not).
 int pick_tile_shift(long long scored_elems, int max_ctas);

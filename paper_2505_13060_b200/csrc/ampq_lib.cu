@@ -104,6 +104,7 @@ struct ampq_ctx {
     std::vector<LayerRec> layers;
     std::vector<Group> groups;
     int scale_pow2 = 0;    // AMPQ_SCALE_POW2: power-of-two scales
+    bool measured = true;  // false: only the model term S is scored (no amax pass, no cast)
     bool amax_ready = false;  // ampq_measure_amax (or a score) has filled the amax mirror
     bool dirty = true;     // bindings changed since the tables were built
     bool scored = false;   // a score has been issued
@@ -619,6 +620,13 @@ int ampq_set_scale_mode(ampq_ctx* ctx, int mode) {
     return AMPQ_OK;
 }
 
+int ampq_set_measured(ampq_ctx* ctx, int on) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    ctx->measured = on != 0;
+    ctx->scored = false;
+    return AMPQ_OK;
+}
+
 int ampq_measure_amax(ampq_ctx* ctx) {
     if (!ctx) return AMPQ_ERR_INVALID;
     DeviceGuard g(ctx->device);
@@ -686,10 +694,12 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[1], st), "cudaEventRecord");
-        if (ctx->namax_tiles > 0) {
+        if (ctx->namax_tiles > 0 && ctx->measured) {
             AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
             ++ctx->launches;
         }
+        if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched
+            AMPQ_CUDA(cudaMemsetAsync(ctx->d_partials.p, 0, (size_t)ctx->nslots * nacc * sizeof(double), st), "memset partials");
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
         AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
         ++ctx->launches;
@@ -698,8 +708,9 @@ int ampq_score(ampq_ctx* ctx) {
             if (ctx->ntiles[c] <= 0) continue;
             const bool causal = c >= 2 * kMaxRB;  // the last two classes: triangular operands, fp32 and bf16
             AMPQ_CUDA(launch_score(causal ? c - 2 * kMaxRB : c / kMaxRB, causal ? 1 : c % kMaxRB + 1, ctx->d_tens.p,
-                                   ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas, ctx->fmask,
-                                   ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st, causal ? 1 : 0), "score");
+                                   ctx->d_tile_begin[c].p, T, ctx->ntiles[c], ctx->tile_shift, ctx->max_ctas,
+                                   ctx->measured ? ctx->fmask : 0, ctx->d_scales.p, ctx->d_partials.p, ctx->d_status.p, st,
+                                   causal ? 1 : 0, nacc), "score");
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");
@@ -811,9 +822,13 @@ int ampq_stream_sample(ampq_ctx* ctx, int layer_id, int operand, int r, int dtyp
     AMPQ_CUDA(ctx->d_job_partials.ensure((size_t)ntiles * nacc + 1), "cudaMalloc(job partials)");
     SegmentJob* job = ctx->d_jobs.p + seg;
     cudaStream_t st = ctx->stream;
-    if ((rc = job_amax_and_scales(ctx, job, dtype, values, grads, numel, l.op[operand].amax_preset, ntiles))) return rc;
+    // S only: a preset of 0 keeps the amax pass away; the D columns of the slots are cleared instead of written
+    const float preset = ctx->measured ? l.op[operand].amax_preset : 0.0f;
+    if ((rc = job_amax_and_scales(ctx, job, dtype, values, grads, numel, preset, ntiles))) return rc;
+    if (!ctx->measured && ntiles > 0)
+        AMPQ_CUDA(cudaMemsetAsync(ctx->d_job_partials.p, 0, (size_t)ntiles * nacc * sizeof(double), st), "memset partials");
     AMPQ_CUDA(launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &job->tensor, job->tile_begin, 1, ntiles, shift, ctx->max_ctas,
-                           ctx->fmask, job->scales, ctx->d_job_partials.p, ctx->d_status.p, st), "score");
+                           ctx->measured ? ctx->fmask : 0, job->scales, ctx->d_job_partials.p, ctx->d_status.p, st, 0, nacc), "score");
     AMPQ_CUDA(launch_finalize(&job->segment, 1, nacc, ctx->d_job_partials.p, ctx->d_seg_out.p + (size_t)seg * nacc, st), "finalize");
     AMPQ_CUDA(launch_job_fold(job, tensor, ctx->d_amax_bits.p, ctx->d_flags.p, ctx->d_scales.p, st), "job_fold");
     ctx->launches += numel > 0 ? 6 : 4;

@@ -505,3 +505,52 @@ def test_random_mix_of_layers_in_one_score(ampq, orc, seed):
     for lid, lt in layers:
         compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, low, threads=8), 1 + len(low), lt.spec.name)
     ctx.destroy()
+
+
+def test_model_term_only(ampq, orc):
+    """ampq_set_measured(0): only S is scored -- equal to the S of the full pass
+    and to the oracle's, with no amax pass, all measured values 0, and the same
+    plan under the paper's own loss-MSE model."""
+    specs = synth.llama7b_block(16)[:4] + synth.toy_mlp(R=3, tokens=50, width=130, layers=2)
+    lts = [synth.make_layer(s, "cuda", seed=23, layer=i) for i, s in enumerate(specs)]
+    full = _ctx(ampq, (0, E4M3, E5M2))
+    only = _ctx(ampq, (0, E4M3, E5M2))
+    only.set_measured(False)
+    fid, oid = _register(ampq, full, lts), _register(ampq, only, lts)
+    full.score()
+    only.score()
+    assert only.last_launch_count() == full.last_launch_count() - 1   # no amax launch
+    rng = np.random.default_rng(3)
+    for a, b, lt in zip(fid, oid, lts):
+        fr, orr = full.get_layer(a), only.get_layer(b)
+        ref = oracle_layer(orc, lt, [E4M3, E5M2])
+        assert orr["s_per_sample"].tobytes() == fr["s_per_sample"].tobytes()
+        assert orr["d_model"].tobytes() == fr["d_model"].tobytes()
+        assert_close(orr["s_per_sample"], ref["s_per_sample"], lt.spec.name + " s^r")
+        assert_close(orr["d_model"], ref["d_model"], lt.spec.name + " d_model")
+        assert not orr["d_meas"].any() and not orr["d_meas_per_sample"].any() and not orr["amax"].any()
+        assert not only.get_operand(b, 0)[:, 1:].any()
+        c = [0.0, float(rng.uniform(0.5, 2.0)), float(rng.uniform(0.5, 2.0))]
+        for cx, lid in ((full, a), (only, b)):
+            cx.define_group([lid], np.array([[0, 1, 2]], np.uint8), c)
+    budget = 0.3 * full.all_lowp_cost(ampq.D_MODEL, 1)
+    pf, po = full.select(ampq.D_MODEL, budget), only.select(ampq.D_MODEL, budget)
+    assert pf[0].tolist() == po[0].tolist() and pf[1:] == po[1:]
+    # streamed, S only
+    only.stream_begin()
+    lt = lts[0]
+    for r in range(lt.spec.R):
+        x, gx = lt.values[0][r], lt.grads[0][r]
+        only.stream_sample(oid[0], 0, r, ampq.BF16, x.data_ptr(), gx.data_ptr(), x.numel())
+    only.stream_end()
+    got = only.get_operand(oid[0], 0)
+    assert_close(got[:, 0], full.get_operand(fid[0], 0)[:, 0], "streamed S", tol=1e-12)
+    assert not got[:, 1:].any()
+    # back to both terms
+    only.set_measured(True)
+    for lid, lt in zip(oid, lts):
+        ampq.bind_layer_tensors(only, lid, lt)
+    only.score()
+    assert only.get_layer(oid[1])["d_meas"].tobytes() == full.get_layer(fid[1])["d_meas"].tobytes()
+    full.destroy()
+    only.destroy()
