@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 # source it was taken on: `kernels_sha256` is the digest of ampq_kernels.cu +
 # ampq_device.h at capture time, and the bench reports traffic = null otherwise.
 NCU_TRAFFIC = {
-    "kernels_sha256": "af743df515b76552c1cbed61fcd435a16f334555fdca2c4e9b50dfbd208a92f5",
-    "dram_bytes_per_scored_byte": {"e4m3": 1.0040},
+    "kernels_sha256": "78f8393fcade63c10e9782290c7e66034749a43747d126d0d57af93f82d29708",
+    "dram_bytes_per_scored_byte": {"e4m3": 1.0045},
     "source": "profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md",
 }
 
