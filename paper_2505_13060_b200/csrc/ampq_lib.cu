@@ -90,6 +90,12 @@ struct PinBuf {
     }
 };
 
+// A typed window into the result arena (see ensure_results).
+template <typename T>
+struct View {
+    T* p = nullptr;
+};
+
 int mantissa_bits_of(int fmt) { return fmt == AMPQ_FMT_E4M3 ? 3 : (fmt == AMPQ_FMT_E5M2 ? 2 : 7); }
 
 }  // namespace
@@ -128,17 +134,19 @@ struct ampq_ctx {
     DevBuf<long long> d_tile_begin[kScoreClasses], d_amax_tile_begin;
     DevBuf<Segment> d_segs;
     DevBuf<Layer> d_lay;
-    DevBuf<unsigned> d_amax_bits;
-    DevBuf<float> d_scales;
     DevBuf<double> d_partials;
-    DevBuf<int> d_flags;
-    DevBuf<double> d_seg_out, d_layer_out;
-    DevBuf<LaunchStatus> d_status;
-    PinBuf<unsigned> h_amax_bits;
-    PinBuf<float> h_scales;
-    PinBuf<int> h_flags;
-    PinBuf<double> h_seg_out, h_layer_out;
-    PinBuf<LaunchStatus> h_status;
+    // Every small result of a pass lives in ONE device arena with ONE pinned host
+    // mirror of the same layout, so that reading a pass back is a single copy:
+    // status | amax_bits[T] | flags[T] | scales[T][2][kMaxLow] | seg_out | layer_out
+    DevBuf<unsigned char> d_arena;
+    PinBuf<unsigned char> h_arena;
+    size_t arena_bytes = 0;  // bytes of the current layout
+    View<LaunchStatus> d_status, h_status;
+    View<unsigned> d_amax_bits, h_amax_bits;
+    View<int> d_flags, h_flags;
+    View<float> d_scales, h_scales;
+    View<double> d_seg_out, h_seg_out, d_layer_out, h_layer_out;
+    DevBuf<LaunchStatus> d_fq_status;  // status word of fake-quantisation calls (outside any pass)
 
     // streaming calibration (ampq_stream_*) and fake quantisation
     bool streaming = false;
@@ -186,6 +194,37 @@ int cuda_fail(ampq_ctx* ctx, cudaError_t e, const char* where) {
 bool layer_ready(const LayerRec& l) { return l.op[0].bound && l.op[1].bound; }
 
 long long extent_of(const LayerRec& l, const Operand& o) { return o.per_sample ? o.numel / l.R : o.numel; }
+
+// Lays the result arena out for T tensors, S segments of nacc doubles and
+// layer_doubles doubles of layer blocks, growing the two allocations if needed.
+// Only called when no pass is pending.
+int ensure_results(ampq_ctx* ctx, size_t T, size_t S, int nacc, size_t layer_doubles) {
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t o_status = 0;
+    const size_t o_amax = up(sizeof(LaunchStatus));
+    const size_t o_flags = o_amax + up(T * sizeof(unsigned));
+    const size_t o_scales = o_flags + up(T * sizeof(int));
+    const size_t o_seg = o_scales + up(T * 2 * kMaxLow * sizeof(float));
+    const size_t o_layer = o_seg + up(S * nacc * sizeof(double));
+    const size_t total = o_layer + up(layer_doubles * sizeof(double));
+    AMPQ_CUDA(ctx->d_arena.ensure(total), "cudaMalloc(results)");
+    AMPQ_CUDA(ctx->h_arena.ensure(total), "cudaMallocHost(results)");
+    ctx->arena_bytes = total;
+    unsigned char *d = ctx->d_arena.p, *h = ctx->h_arena.p;
+    ctx->d_status.p = reinterpret_cast<LaunchStatus*>(d + o_status);
+    ctx->h_status.p = reinterpret_cast<LaunchStatus*>(h + o_status);
+    ctx->d_amax_bits.p = reinterpret_cast<unsigned*>(d + o_amax);
+    ctx->h_amax_bits.p = reinterpret_cast<unsigned*>(h + o_amax);
+    ctx->d_flags.p = reinterpret_cast<int*>(d + o_flags);
+    ctx->h_flags.p = reinterpret_cast<int*>(h + o_flags);
+    ctx->d_scales.p = reinterpret_cast<float*>(d + o_scales);
+    ctx->h_scales.p = reinterpret_cast<float*>(h + o_scales);
+    ctx->d_seg_out.p = reinterpret_cast<double*>(d + o_seg);
+    ctx->h_seg_out.p = reinterpret_cast<double*>(h + o_seg);
+    ctx->d_layer_out.p = reinterpret_cast<double*>(d + o_layer);
+    ctx->h_layer_out.p = reinterpret_cast<double*>(h + o_layer);
+    return AMPQ_OK;
+}
 
 // log2 T when the operand may be scored as a stack of lower-triangular T x T
 // matrices, else 0 (scored densely, which gives the same sums).  The triangular
@@ -324,19 +363,11 @@ int upload_tables(ampq_ctx* ctx) {
     AMPQ_CUDA(ctx->d_amax_tile_begin.ensure(T + 1), "cudaMalloc(amax_tile_begin)");
     AMPQ_CUDA(ctx->d_segs.ensure(S), "cudaMalloc(segments)");
     AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
-    AMPQ_CUDA(ctx->d_amax_bits.ensure(T), "cudaMalloc(amax)");
-    AMPQ_CUDA(ctx->d_scales.ensure(T * 2 * kMaxLow), "cudaMalloc(scales)");
-    AMPQ_CUDA(ctx->d_flags.ensure(T), "cudaMalloc(flags)");
     AMPQ_CUDA(ctx->d_partials.ensure((size_t)ctx->nslots * nacc), "cudaMalloc(partials)");
-    AMPQ_CUDA(ctx->d_seg_out.ensure(S * nacc), "cudaMalloc(seg_out)");
-    AMPQ_CUDA(ctx->d_layer_out.ensure((size_t)ctx->layer_out_doubles), "cudaMalloc(layer_out)");
-    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
-    AMPQ_CUDA(ctx->h_amax_bits.ensure(T), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_scales.ensure(T * 2 * kMaxLow), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_flags.ensure(T), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_seg_out.ensure(S * nacc), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_layer_out.ensure((size_t)ctx->layer_out_doubles), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_status.ensure(1), "cudaMallocHost");
+    {
+        const int rc = ensure_results(ctx, T, S, nacc, (size_t)ctx->layer_out_doubles);
+        if (rc) return rc;
+    }
     cudaStream_t st = ctx->stream;
     if (T) {
         AMPQ_CUDA(cudaMemcpyAsync(ctx->d_tens.p, ctx->tens.data(), T * sizeof(Tensor), cudaMemcpyHostToDevice, st), "H2D tensors");
@@ -456,24 +487,21 @@ int combine_and_read_back(ampq_ctx* ctx, int T, int L, int S) {
     }
     AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, prm, ctx->d_seg_out.p, ctx->d_layer_out.p, st), "combine");
     ++ctx->launches;
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_scales.p, ctx->d_scales.p, (size_t)T * 2 * kMaxLow * sizeof(float), cudaMemcpyDeviceToHost, st), "D2H scales");
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_flags.p, ctx->d_flags.p, T * sizeof(int), cudaMemcpyDeviceToHost, st), "D2H flags");
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_seg_out.p, ctx->d_seg_out.p, (size_t)S * nacc * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H segments");
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_layer_out.p, ctx->d_layer_out.p, (size_t)ctx->layer_out_doubles * sizeof(double), cudaMemcpyDeviceToHost, st), "D2H layers");
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_status.p, ctx->d_status.p, sizeof(LaunchStatus), cudaMemcpyDeviceToHost, st), "D2H status");
+    (void)T;
+    (void)S;
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_arena.p, ctx->d_arena.p, ctx->arena_bytes, cudaMemcpyDeviceToHost, st), "D2H results");
     return AMPQ_OK;
 }
 
 // Runs one (tensor, sample) job through amax / scales on the stream; the
 // caller launches what follows.  job is a device pointer.
-int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, int dtype, const void* values, const void* grads,
-                        long long numel, float preset, long long ntiles) {
+int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, LaunchStatus* status, int dtype, const void* values,
+                        const void* grads, long long numel, float preset, long long ntiles) {
     cudaStream_t st = ctx->stream;
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
     AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, st), "job_prepare");
     AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st), "amax");
-    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, ctx->d_status.p, st, ctx->scale_pow2), "scales");
+    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, status, st, ctx->scale_pow2), "scales");
     return AMPQ_OK;
 }
 
@@ -532,12 +560,9 @@ int ampq_destroy(ampq_ctx* ctx) {
                 if (l.op[k].stage) cudaFree(l.op[k].stage);
         ctx->d_tens.release(); ctx->d_amax_tile_begin.release();
         for (auto& b : ctx->d_tile_begin) b.release();
-        ctx->d_segs.release(); ctx->d_lay.release(); ctx->d_amax_bits.release(); ctx->d_scales.release();
-        ctx->d_partials.release(); ctx->d_flags.release(); ctx->d_seg_out.release();
-        ctx->d_layer_out.release(); ctx->d_status.release();
+        ctx->d_segs.release(); ctx->d_lay.release(); ctx->d_partials.release();
+        ctx->d_arena.release(); ctx->h_arena.release(); ctx->d_fq_status.release();
         ctx->d_jobs.release(); ctx->d_job_partials.release(); ctx->d_fq_job.release();
-        ctx->h_amax_bits.release(); ctx->h_scales.release(); ctx->h_flags.release();
-        ctx->h_seg_out.release(); ctx->h_layer_out.release(); ctx->h_status.release();
         for (int i = 0; i < 6; ++i)
             if (ctx->ev[i]) cudaEventDestroy(ctx->ev[i]);
     }
@@ -766,19 +791,11 @@ int ampq_stream_begin(ampq_ctx* ctx) {
     const size_t T = ctx->tens.size(), L = ctx->lay.size(), S = (size_t)nseg;
     const int nacc = ctx->F;
     AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
-    AMPQ_CUDA(ctx->d_amax_bits.ensure(T), "cudaMalloc(amax)");
-    AMPQ_CUDA(ctx->d_scales.ensure(T * 2 * kMaxLow), "cudaMalloc(scales)");
-    AMPQ_CUDA(ctx->d_flags.ensure(T), "cudaMalloc(flags)");
-    AMPQ_CUDA(ctx->d_seg_out.ensure(S * nacc), "cudaMalloc(seg_out)");
-    AMPQ_CUDA(ctx->d_layer_out.ensure((size_t)out_off), "cudaMalloc(layer_out)");
-    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
     AMPQ_CUDA(ctx->d_jobs.ensure(S), "cudaMalloc(jobs)");
-    AMPQ_CUDA(ctx->h_amax_bits.ensure(T), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_scales.ensure(T * 2 * kMaxLow), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_flags.ensure(T), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_seg_out.ensure(S * nacc), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_layer_out.ensure((size_t)out_off), "cudaMallocHost");
-    AMPQ_CUDA(ctx->h_status.ensure(1), "cudaMallocHost");
+    {
+        const int rc = ensure_results(ctx, T, S, nacc, (size_t)out_off);
+        if (rc) return rc;
+    }
     cudaStream_t st = ctx->stream;
     if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
     if (T) {
@@ -824,7 +841,7 @@ int ampq_stream_sample(ampq_ctx* ctx, int layer_id, int operand, int r, int dtyp
     cudaStream_t st = ctx->stream;
     // S only: a preset of 0 keeps the amax pass away; the D columns of the slots are cleared instead of written
     const float preset = ctx->measured ? l.op[operand].amax_preset : 0.0f;
-    if ((rc = job_amax_and_scales(ctx, job, dtype, values, grads, numel, preset, ntiles))) return rc;
+    if ((rc = job_amax_and_scales(ctx, job, ctx->d_status.p, dtype, values, grads, numel, preset, ntiles))) return rc;
     if (!ctx->measured && ntiles > 0)
         AMPQ_CUDA(cudaMemsetAsync(ctx->d_job_partials.p, 0, (size_t)ntiles * nacc * sizeof(double), st), "memset partials");
     AMPQ_CUDA(launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &job->tensor, job->tile_begin, 1, ntiles, shift, ctx->max_ctas,
@@ -866,8 +883,9 @@ int ampq_fake_quant(ampq_ctx* ctx, int dtype, int fmt, const void* values, long 
     DeviceGuard g(ctx->device);
     if (!g.ok) return fail(ctx, AMPQ_ERR_CUDA, "cudaSetDevice failed");
     AMPQ_CUDA(ctx->d_fq_job.ensure(1), "cudaMalloc(job)");
-    AMPQ_CUDA(ctx->d_status.ensure(1), "cudaMalloc(status)");
-    int rc = job_amax_and_scales(ctx, ctx->d_fq_job.p, dtype, values, values, numel, amax >= 0.0f ? amax : -1.0f, 0);
+    AMPQ_CUDA(ctx->d_fq_status.ensure(1), "cudaMalloc(status)");
+    int rc = job_amax_and_scales(ctx, ctx->d_fq_job.p, ctx->d_fq_status.p, dtype, values, values, numel,
+                                 amax >= 0.0f ? amax : -1.0f, 0);
     if (rc) return rc;
     const float* pair = ctx->d_fq_job.p->scales + ctx->slot_of_fmt[f] * 2;
     AMPQ_CUDA(launch_fake_quant(dtype, fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2, values, numel, pair, dev_out, ctx->stream), "fake_quant");
