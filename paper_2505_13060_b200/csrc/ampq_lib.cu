@@ -798,13 +798,8 @@ int ampq_stream_begin(ampq_ctx* ctx) {
     }
     cudaStream_t st = ctx->stream;
     if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
-    if (T) {
-        AMPQ_CUDA(cudaMemsetAsync(ctx->d_amax_bits.p, 0, T * sizeof(unsigned), st), "memset amax");
-        AMPQ_CUDA(cudaMemsetAsync(ctx->d_flags.p, 0, T * sizeof(int), st), "memset flags");
-        AMPQ_CUDA(cudaMemsetAsync(ctx->d_scales.p, 0, T * 2 * kMaxLow * sizeof(float), st), "memset scales");
-    }
-    if (S) AMPQ_CUDA(cudaMemsetAsync(ctx->d_seg_out.p, 0, S * nacc * sizeof(double), st), "memset seg_out");
-    AMPQ_CUDA(cudaMemsetAsync(ctx->d_status.p, 0, sizeof(LaunchStatus), st), "memset status");
+    // amax, flags, scales, every per-sample sum and the status word start at zero
+    AMPQ_CUDA(cudaMemsetAsync(ctx->d_arena.p, 0, ctx->arena_bytes, st), "memset results");
     ctx->streaming = true;
     ctx->scored = false;
     ctx->dirty = true;  // a later ampq_score rebuilds its own tables
