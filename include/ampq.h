@@ -102,7 +102,8 @@ int ampq_register_layer(ampq_ctx *ctx, int kind, const char *name, int R, int *l
  * to the element size (AMPQ_ERR_ALIGN otherwise); 16-byte alignment of every
  * sample slice enables the vectorised path, anything else is scored
  * correctly through a slower scalar path.  numel = 0 is allowed (scores 0).
- * Re-binding replaces the previous binding. */
+ * Re-binding replaces the previous binding.  Several layers may bind the very
+ * same values (layers that read one input): its amax is then measured once. */
 int ampq_bind_operand(ampq_ctx *ctx, int layer_id, int operand, int dtype, int mem,
                       const void *values, long long numel, int per_sample_values,
                       const void *grads, long long grad_stride);

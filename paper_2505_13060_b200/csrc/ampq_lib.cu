@@ -128,6 +128,7 @@ struct ampq_ctx {
     std::vector<Layer> lay;
     std::vector<int> scored_layer_ids;
     long long ntiles[kScoreClasses] = {}, namax_tiles = 0, nslots = 0;
+    std::vector<std::pair<int, int>> amax_alias;  // (tensor, earlier tensor bound to the very same values)
     int layer_out_doubles = 0;
 
     DevBuf<Tensor> d_tens;
@@ -245,12 +246,13 @@ int causal_shift_of(const LayerRec& l, const Operand& o, const Tensor& t) {
 
 // Builds the host tables for every layer whose two operands are bound.
 int build_tables(ampq_ctx* ctx) {
-    ctx->tens.clear(); ctx->amax_tile_begin.clear();
+    ctx->tens.clear(); ctx->amax_tile_begin.clear(); ctx->amax_alias.clear();
     for (auto& tb : ctx->tile_begin) tb.clear();
     ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
     for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
     long long tiles[kScoreClasses] = {}, atiles = 0, slots = 0;
     int out_off = 0;
+    std::vector<char> measures_amax;  // per tensor: it has amax tiles of its own
     long long scored_elems = 0;  // value elements the scoring launches walk (shared values once per sample group)
     for (const auto& l : ctx->layers) {
         if (!layer_ready(l)) continue;
@@ -317,13 +319,28 @@ int build_tables(ampq_ctx* ctx) {
                 my_tiles[c0 + kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
                 if (l.R % kMaxRB) my_tiles[c0 + l.R % kMaxRB - 1] += t.tiles_per_seg;
             }
-            const long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
+            long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
+            // Layers that read the same tensor (q, k, v or gate, up of one block share
+            // their input) need its amax only once: a later binding of the very same
+            // device values takes the amax of the first instead of another read.
+            if (my_atiles > 0 && o.mem == AMPQ_MEM_DEVICE) {
+                for (size_t e = 0; e < ctx->tens.size(); ++e) {
+                    const Tensor& u = ctx->tens[e];
+                    if (measures_amax[e] && u.values == t.values && u.numel == t.numel && u.dtype == t.dtype &&
+                        u.causal_shift == t.causal_shift) {
+                        ctx->amax_alias.emplace_back((int)ctx->tens.size(), (int)e);
+                        my_atiles = 0;
+                        break;
+                    }
+                }
+            }
             for (int c = 0; c < kScoreClasses; ++c) {
                 ctx->tile_begin[c].push_back(tiles[c]);
                 tiles[c] += my_tiles[c];
             }
             ctx->amax_tile_begin.push_back(atiles);
             atiles += my_atiles;
+            measures_amax.push_back(my_atiles > 0);
             for (int r = 0; r < l.R; ++r) {
                 Segment s{};
                 s.first_slot = slots + (long long)r * t.tiles_per_seg;
@@ -472,6 +489,14 @@ int prepare_tables(ampq_ctx* ctx) {
         if ((rc = upload_tables(ctx))) return rc;
         ctx->dirty = false;
     }
+    return AMPQ_OK;
+}
+
+// Tensors bound to the same values as an earlier one take that one's amax.
+int copy_alias_amax(ampq_ctx* ctx) {
+    for (const auto& a : ctx->amax_alias)
+        AMPQ_CUDA(cudaMemcpyAsync(ctx->d_amax_bits.p + a.first, ctx->d_amax_bits.p + a.second, sizeof(unsigned),
+                                  cudaMemcpyDeviceToDevice, ctx->stream), "D2D amax");
     return AMPQ_OK;
 }
 
@@ -668,6 +693,7 @@ int ampq_measure_amax(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
         AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
         ctx->launches = ctx->namax_tiles > 0 ? 2 : 1;
+        if ((rc = copy_alias_amax(ctx))) return rc;
         AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
     }
     ctx->amax_ready = true;
@@ -722,6 +748,7 @@ int ampq_score(ampq_ctx* ctx) {
         if (ctx->namax_tiles > 0 && ctx->measured) {
             AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
             ++ctx->launches;
+            if ((rc = copy_alias_amax(ctx))) return rc;
         }
         if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched
             AMPQ_CUDA(cudaMemsetAsync(ctx->d_partials.p, 0, (size_t)ctx->nslots * nacc * sizeof(double), st), "memset partials");

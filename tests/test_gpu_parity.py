@@ -554,3 +554,29 @@ def test_model_term_only(ampq, orc):
     assert only.get_layer(oid[1])["d_meas"].tobytes() == full.get_layer(fid[1])["d_meas"].tobytes()
     full.destroy()
     only.destroy()
+
+
+def test_layers_sharing_one_input_tensor(ampq, orc):
+    """q, k, v of a block read the same activations: three layers bound to the
+    very same values (with their own gradients and weights) get the amax of the
+    first binding without another read, and every value still equals the
+    oracle's; a preset on one of them or different extents break the sharing."""
+    specs = synth.llama7b_block(16)[:3]
+    lts = [synth.make_layer(s, "cuda", seed=31, layer=i) for i, s in enumerate(specs)]
+    for lt in lts[1:]:
+        lt.values[0] = lts[0].values[0]   # one X for all three
+    lts[0].values[0][1, 5, 7] = 300.0   # an amax that only a real read of X can find
+    ctx = _ctx(ampq, (0, E4M3))
+    ids = _register(ampq, ctx, lts)
+    ctx.score()
+    refs = [oracle_layer(orc, lt, [E4M3]) for lt in lts]
+    for lid, lt, ref in zip(ids, lts, refs):
+        got = compare_layer(ampq, ctx, lid, ref, 2, "shared input " + lt.spec.name)
+        assert got["amax"][0] == np.float32(300.0)
+    ctx.measure_amax()
+    assert all(ctx.get_amax(i)[0] == np.float32(300.0) for i in ids)
+    ctx.set_amax(ids[1], 0, 2.0)   # a preset on one sibling: the others still measure
+    ctx.score()
+    compare_layer(ampq, ctx, ids[1], oracle_layer(orc, lts[1], [E4M3], amax_presets=(2.0, None)), 2, "preset sibling")
+    compare_layer(ampq, ctx, ids[2], refs[2], 2, "unpreset sibling")
+    ctx.destroy()
