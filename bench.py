@@ -9,7 +9,16 @@ weighting / reduction, ordered finalize and the per-layer combine, for
 once, so block b is bound to device slot b mod ``--resident-blocks`` (each slot
 is a full block of distinct random tensors, 7.68 GB); two passes over a slot are
 tens of GB of other traffic apart, far beyond the 126 MB L2, so every byte
-comes from HBM.
+comes from HBM.  Because the slots stand for different blocks, the library's
+pointer-based sharing (one amax pass and one read for layers bound to the very
+same values) is switched off for these bindings: every one of the 1120 operands
+is measured and scored in full.  A line whose byte rates exceed 1.2 x the
+measured HBM peak reports ``value: null`` with the reason.
+
+``--gpus N`` started as a plain process starts the N ranks itself (torchrun on
+127.0.0.1).  Ranks are independent replicas by default; ``--shard layers``
+splits one model's layers over the ranks and adds the table exchange and the
+selection to the step.
 
 Prints one JSON line: ``value`` = scored bytes of all ranks / device time of the
 step (CUDA events, max over ranks); ``roofline`` for the scoring kernel from
@@ -66,6 +75,14 @@ def parse_args():
                     help="side measurement: score only the paper's model term S (no amax pass, no FP8 cast)")
     ap.add_argument("--causal", action="store_true",
                     help="attention workload: declare the softmax operand causal so that its zero triangle is not read")
+    ap.add_argument("--shared-inputs", action="store_true",
+                    help="side measurement (llama70b / llama7b): q,k,v bind one input tensor and gate,up another, as "
+                         "in a real transformer block, each layer with gradients of its own; every block is resident "
+                         "(no slot reuse), and the library reads each shared input once")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "layers"],
+                    help="several ranks: 'replicas' gives every rank its own copy of the workload (weak scaling, no "
+                         "exchange); 'layers' splits ONE model's layers over the ranks, exchanges the per-layer table "
+                         "and runs the sub-graph sums and the selection on every rank (strong scaling)")
     ap.add_argument("--layers", default="",
                     help="comma-separated subset of a block's layers (q,k,v,o,gate,up,down); a small case of the "
                          "same kernels for profiler captures, never the benchmark")
@@ -260,24 +277,38 @@ def workload_specs(workload: str, layers: str = ""):
     return specs
 
 
-def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int, causal: bool = False):
+def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int, causal: bool = False,
+                  shared_inputs: bool = False, only=None):
     """Registers `blocks` blocks of `specs` in ctx.  Block b is bound to device
     slot b mod nres; each slot is a full block of distinct random tensors.
+    The slots stand for `blocks` different blocks, so the library is told NOT to
+    treat equal pointers as one tensor (ampq_set_sharing off): every binding is
+    measured and scored in full.  With `shared_inputs` (needs blocks == nres)
+    q,k,v and gate,up of a block bind one input each and sharing stays on.
     With `causal`, causal-softmax operands are declared triangular and only the
-    bytes on or left of the diagonal count as scored.
+    bytes on or left of the diagonal count as scored.  `only`: the set of global
+    layer indices (block * len(specs) + i) this process registers.
     Returns (slots, layer ids, scored bytes of one score)."""
     import torch
 
     from paper_2505_13060_b200 import binding as ampq
     from paper_2505_13060_b200 import synth
 
+    if shared_inputs and blocks != nres:
+        raise SystemExit("--shared-inputs needs every block resident")
+    ctx.set_sharing(shared_inputs)
     slots = []
     for s in range(nres):
-        slots.append([synth.make_layer(sp, dev, seed=seed, layer=len(specs) * s + i) for i, sp in enumerate(specs)])
+        lts = [synth.make_layer(sp, dev, seed=seed, layer=len(specs) * s + i) for i, sp in enumerate(specs)]
+        if shared_inputs:
+            synth.share_block_inputs(lts)
+        slots.append(lts)
     torch.cuda.synchronize()
     ids, scored_bytes = [], 0
     for b in range(blocks):
         for i, sp in enumerate(specs):
+            if only is not None and b * len(specs) + i not in only:
+                continue
             lid = ctx.register_layer(sp.kind, "blk%d.%s" % (b, sp.name), sp.R)
             ampq.bind_layer_tensors(ctx, lid, slots[b % nres][i])
             ids.append(lid)
@@ -291,11 +322,26 @@ def bind_workload(ctx, specs, blocks: int, nres: int, dev, seed: int, causal: bo
     return slots, ids, scored_bytes
 
 
+def selection_groups(specs, blocks: int, seed: int = 0):
+    """One sub-graph per block with two configurations, all layers in the
+    baseline format or all in the low-precision one (the benchmark's per-block
+    groups); gains drawn uniformly in [0.5, 2] ms.  Layer indices are global."""
+    import numpy as np
+
+    rng = np.random.default_rng(seed)
+    n = len(specs)
+    groups = []
+    for b in range(blocks):
+        Q = np.array([[0, 1]] * n, dtype=np.uint8)
+        groups.append((list(range(b * n, (b + 1) * n)), Q, np.array([0.0, rng.uniform(0.5, 2.0)])))
+    return groups
+
+
 def run_b200(args):
     import torch
 
     from paper_2505_13060_b200 import binding as ampq
-    from paper_2505_13060_b200 import synth
+    from paper_2505_13060_b200 import shard, synth
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -311,17 +357,30 @@ def run_b200(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
     fmts = {"e4m3": [0, 1], "e5m2": [0, 2], "both": [0, 1, 2]}[args.formats]
+    F = len(fmts)
+    shard_layers = args.shard == "layers"
 
     specs = workload_specs(args.workload, args.layers)
     block_gb = sum(sp.scored_bytes() for sp in specs) / 1e9
     nres = max(1, min(args.resident_blocks, args.blocks))
+    if args.shared_inputs:
+        args.blocks = nres
     stream = torch.cuda.Stream(device=dev)
     ctx = ampq.Context(local_rank, stream.cuda_stream)
     ctx.set_formats(fmts)
     if args.model_only:
         ctx.set_measured(False)
-    slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev, seed=100 + rank, causal=args.causal)
-    value_bytes = args.blocks * sum(sp.value_bytes() for sp in specs)
+    n_layers_model = args.blocks * len(specs)
+    only, owner = None, None
+    if shard_layers:
+        # ONE model: its layers are dealt to the ranks by scored bytes, the same way on every rank
+        owner = shard.assign_layers([sp.scored_bytes() for _ in range(args.blocks) for sp in specs], world)
+        only = {i for i in range(n_layers_model) if owner[i] == rank}
+    slots, ids, scored_bytes = bind_workload(ctx, specs, args.blocks, nres, dev,
+                                             seed=100 + (0 if shard_layers else rank), causal=args.causal,
+                                             shared_inputs=args.shared_inputs, only=only)
+    my_global = sorted(only) if only is not None else list(range(n_layers_model))
+    groups = selection_groups(specs, args.blocks) if shard_layers else None
     ctx.set_timing(True)
 
     def barrier():
@@ -329,10 +388,27 @@ def run_b200(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    plan = None
+
+    def step():
+        """One pass of the hot path.  Layer-sharded: plus the exchange of the
+        per-layer table and the sub-graph sums and selection on every rank."""
+        nonlocal plan
         ctx.score()
+        t = ctx.get_timing()  # synchronises the step; the per-kernel events are the library's own
+        if shard_layers:
+            rows = {g: shard.layer_row(ctx.get_layer(lid), F) for g, lid in zip(my_global, ids)}
+            table = shard.gather_layer_table(rows, n_layers_model, F, device=dev)
+            all_low = float(table[:, 1 + F + 1].sum())
+            plan = shard.select_from_table(ampq, table, F, groups, ampq.D_MEASURED, 0.2 * all_low)
+        return t
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
     ctx.get_layer(ids[0])
     launches_per_step = ctx.last_launch_count()
+    pass_bytes = ctx.get_pass_bytes()
     sampler = ClockSampler(local_rank) if rank == 0 else None
     ev0 = torch.cuda.Event(enable_timing=True)
     ev1 = torch.cuda.Event(enable_timing=True)
@@ -343,36 +419,42 @@ def run_b200(args):
     with torch.cuda.stream(stream):
         ev0.record(stream)
         for _ in range(args.steps):
-            ctx.score()
-            t = ctx.get_timing()  # synchronises the step; the per-kernel events are the library's own
+            t = step()
             score_ms.append(t["score_ms"])
             amax_ms.append(t["amax_ms"])
         ev1.record(stream)
     barrier()
     clocks = sampler.stop() if sampler else None
     total_ms = ev0.elapsed_time(ev1)
+    job_scored_bytes = world * scored_bytes
     if dist is not None:
         tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
+        if shard_layers:
+            sb = torch.tensor([float(scored_bytes)], device=dev, dtype=torch.float64)
+            dist.all_reduce(sb, op=dist.ReduceOp.SUM)
+            job_scored_bytes = int(sb.item())
     ms_per_step = total_ms / args.steps
-    value = world * scored_bytes / (ms_per_step * 1e-3) / 1e9
+    value = job_scored_bytes / (ms_per_step * 1e-3) / 1e9
     first = ctx.get_layer(ids[0])
 
-    # ---- roofline of the dominant kernel (the fused scoring kernel)
+    # ---- roofline of the dominant kernel (the fused scoring kernel) on this rank
     peak, peak_kind = hbm_peak()
     k_ms = sum(score_ms) / len(score_ms)
+    a_ms = sum(amax_ms) / len(amax_ms)
     achieved = scored_bytes / (k_ms * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "score_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_source": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured" else "fallback 6650 GB/s",
         "traffic": None, "kernel_ms": k_ms, "algorithmic_bytes_per_launch": scored_bytes,
-        "amax_kernel_ms": sum(amax_ms) / len(amax_ms),
-        "amax_kernel_gbs": value_bytes / (sum(amax_ms) / len(amax_ms) * 1e-3) / 1e9,
+        "bytes_read_by_scoring_launches": pass_bytes["score"],
+        "amax_kernel_ms": a_ms, "amax_bytes_read": pass_bytes["amax"],
+        "amax_kernel_gbs": pass_bytes["amax"] / (a_ms * 1e-3) / 1e9 if a_ms > 0 else None,
         "frac_of_8000_datasheet": achieved / 8000.0,
     }
     ratio = NCU_TRAFFIC["dram_bytes_per_scored_byte"].get(args.formats)
-    if ratio is not None and kernels_digest() == NCU_TRAFFIC["kernels_sha256"]:
+    if ratio is not None and kernels_digest() == NCU_TRAFFIC["kernels_sha256"] and not args.shared_inputs and not args.causal:
         roofline["traffic"] = ratio * scored_bytes  # scaled from the small capture to this launch
         roofline["traffic_source"] = NCU_TRAFFIC["source"]
 
@@ -413,7 +495,8 @@ def run_b200(args):
         for sp in specs:
             d2h += 8 * (sp.R + 1 + sp.R * len(fmts) + 2 * len(fmts)) + 2 * (4 + 16 + 4) + 2 * 8 * sp.R * len(fmts)
         e_ms = a0.elapsed_time(a1) / args.e2e_steps
-        assert res[0]["s_mean"] == ctx.get_layer(ids[0])["s_mean"]
+        if my_global[0] == 0 and not args.causal:   # same tensors, another tiling: equal up to the order of the fp64 additions
+            assert abs(res[0]["s_mean"] - first["s_mean"]) <= 1e-9 * abs(first["s_mean"])
         e2e = {"value": block_scored / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e_ms,
                "workload": "one %s-shaped block per step from pinned host memory (AMPQ_MEM_HOST binding)" % args.workload}
@@ -421,6 +504,8 @@ def run_b200(args):
         del host_layers
 
     check = {"s_mean_layer0": first["s_mean"], "d_meas_layer0": float(first["d_meas"][1])}
+    if plan is not None:
+        check["plan_low_precision_groups"] = int(plan[0].sum())
     ctx.destroy()
     del slots
     torch.cuda.empty_cache()
@@ -435,36 +520,69 @@ def run_b200(args):
                "sample": desc + ", %.2f GB scored in %.1f s" % (nbytes / 1e9, dt)}
 
     if rank == 0:
+        read_bytes = pass_bytes["amax"] + pass_bytes["score"]   # what this rank's step reads from HBM
+        whole_gbs = read_bytes / (ms_per_step * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "strong" if shard_layers else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else "") + ("[causal]" if args.causal else "") + ("[model term only]" if args.model_only else ""), "blocks": args.blocks, "layers": len(ids), "R": specs[0].R,
+                "workload": args.workload + "_shaped" + ("[%s]" % args.layers if args.layers else "") + ("[causal]" if args.causal else "")
+                            + ("[model term only]" if args.model_only else "") + ("[q,k,v and gate,up share their input]" if args.shared_inputs else ""),
+                "blocks": args.blocks, "layers": n_layers_model, "layers_on_rank0": len(ids), "R": specs[0].R,
                 "tokens_per_sample": specs[0].op0.shape[-2], "operand_dtype": "bf16", "formats": args.formats,
                 "scored_bytes_per_step_per_gpu": scored_bytes, "resident_blocks": nres,
-                "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block" % (nres, block_gb),
+                "residency": "block b reads device slot b %% %d; each slot is a distinct %.2f GB block; the library "
+                             "treats every binding as a tensor of its own (pointer sharing off)" % (nres, block_gb)
+                             if not args.shared_inputs else "every block resident, pointer sharing on",
                 "l2": "inputs larger than L2 (%.1f GB resident, 126 MB L2)" % (nres * block_gb),
-                "parallelism": "independent layers per GPU, no data-path collective",
+                "parallelism": ("one model, layers dealt to %d ranks by scored bytes; per-layer table exchanged by one "
+                                "all-reduce; sub-graph sums and selection on every rank" % world) if shard_layers
+                               else "independent replicas per GPU, no data-path collective",
             },
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu,
             "check": check,
-            "pct_of_hbm_peak": {"measured_%.0f" % peak: 100.0 * value / peak, "datasheet_8000": 100.0 * value / 8000.0},
-            # every byte the step reads (the amax pass reads each operand once more), all ranks
-            "whole_pass_traffic": {"algorithmic_bytes_per_gpu": scored_bytes + value_bytes,
-                                   "gbs": world * (scored_bytes + value_bytes) / (ms_per_step * 1e-3) / 1e9,
-                                   "frac_of_measured_peak": (scored_bytes + value_bytes) / (ms_per_step * 1e-3) / 1e9 / peak},
+            "pct_of_hbm_peak": {"measured_%.0f" % peak: 100.0 * value / peak / world, "datasheet_8000": 100.0 * value / 8000.0 / world},
+            # every byte the step reads on rank 0 (the amax pass reads each operand once more)
+            "whole_pass_traffic": {"bytes_read_per_gpu": read_bytes, "gbs": whole_gbs, "frac_of_measured_peak": whole_gbs / peak},
         }
+        # A step cannot read HBM much faster than the measured copy peak: such a
+        # number means the timed region skipped work, so it is not reported.
+        limit = 1.2 * peak
+        too_fast = [k for k, v in (("whole_pass_traffic.gbs", whole_gbs), ("roofline.amax_kernel_gbs", roofline["amax_kernel_gbs"]),
+                                   ("roofline.achieved (bytes read)", pass_bytes["score"] / (k_ms * 1e-3) / 1e9))
+                    if v is not None and v > limit]
+        if too_fast:
+            line["rejected_value"] = value
+            line["value"] = None
+            line["invalid"] = "implausible: %s above 1.2 x the measured HBM peak (%.0f GB/s)" % (", ".join(too_fast), limit)
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def relaunch_ranks(args):
+    """`--gpus N` (N > 1) started as a plain process: start the N ranks with
+    torchrun on this node and let them print the line."""
+    import socket
+
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
 
 
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        relaunch_ranks(args)
     else:
         run_b200(args)
 

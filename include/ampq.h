@@ -103,7 +103,7 @@ int ampq_register_layer(ampq_ctx *ctx, int kind, const char *name, int R, int *l
  * sample slice enables the vectorised path, anything else is scored
  * correctly through a slower scalar path.  numel = 0 is allowed (scores 0).
  * Re-binding replaces the previous binding.  Several layers may bind the very
- * same values (layers that read one input): its amax is then measured once. */
+ * same values (layers that read one input); see ampq_set_sharing. */
 int ampq_bind_operand(ampq_ctx *ctx, int layer_id, int operand, int dtype, int mem,
                       const void *values, long long numel, int per_sample_values,
                       const void *grads, long long grad_stride);
@@ -143,6 +143,18 @@ int ampq_set_scale_mode(ampq_ctx *ctx, int mode);
  * detected up front: it shows as a non-finite S.  on = 1 (default): both terms.
  * Applies to ampq_score and ampq_stream_sample. */
 int ampq_set_measured(ampq_ctx *ctx, int on);
+
+/* Layers that read one input (q, k, v or gate, up of a transformer block) bind
+ * the very same values pointer with gradients of their own: z is shared, the
+ * per-layer sensitivity s_l^r = ||z (.) dz||^2 of Sec. 2.2 differs only in the
+ * gradient.  With sharing on (the default) the library recognises such
+ * bindings by pointer, size, dtype, R, gradient stride and preset: the amax of
+ * the values is measured once, and up to four such per-sample operands are
+ * scored in one read and one FP8 cast of the values with one gradient stream
+ * per layer.  Results are those of separate scoring up to the order of the
+ * fp64 additions.  on = 0 treats every binding as a tensor of its own -- for
+ * callers that re-use one buffer for unrelated layers' bindings. */
+int ampq_set_sharing(ampq_ctx *ctx, int on);
 
 /* Only the first step of ampq_score: amax of every bound operand of every fully
  * bound layer (preset ones keep their preset), asynchronously on the stream.
@@ -208,6 +220,15 @@ int ampq_fake_quant(ampq_ctx *ctx, int dtype, int fmt, const void *values, long 
 
 /* Number of kernel launches issued by the last ampq_score (diagnostics). */
 int ampq_last_launch_count(const ampq_ctx *ctx);
+
+/* Bytes of the bound tensors that the last ampq_score (or ampq_measure_amax)
+ * reads (diagnostics; host pointer, bytes[2]): bytes[0] the amax pass -- every
+ * operand without a preset once, an operand several layers share once;
+ * bytes[1] the scoring pass -- values and gradients as the kernels walk them:
+ * shared values (weights) once per group of up to four samples, an input shared
+ * by several layers once per group, triangular operands only up to the
+ * diagonal. */
+int ampq_get_pass_bytes(ampq_ctx *ctx, long long *bytes);
 
 /* Optional device timing of the kernels of a score.  With timing on, ampq_score
  * records CUDA events on its stream around the amax kernel, the scoring kernel

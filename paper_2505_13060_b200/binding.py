@@ -38,6 +38,7 @@ EXPORTS = [
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
     "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal", "ampq_set_measured",
+    "ampq_set_sharing", "ampq_get_pass_bytes",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -88,6 +89,8 @@ def lib():
     L.ampq_fake_quant.argtypes = [vp, i, i, vp, ll, C.c_float, vp]
     L.ampq_set_causal.argtypes = [vp, i, i, ll]
     L.ampq_set_measured.argtypes = [vp, i]
+    L.ampq_set_sharing.argtypes = [vp, i]
+    L.ampq_get_pass_bytes.argtypes = [vp, vp]
     L.ampq_set_scale_mode.argtypes = [vp, i]
     L.ampq_measure_amax.argtypes = [vp]
     L.ampq_get_amax.argtypes = [vp, i, vp]
@@ -269,6 +272,9 @@ class Context:
     def set_measured(self, on: bool):
         self._check(lib().ampq_set_measured(self._h, 1 if on else 0))
 
+    def set_sharing(self, on: bool):
+        self._check(lib().ampq_set_sharing(self._h, 1 if on else 0))
+
     def set_scale_mode(self, mode: int):
         self._check(lib().ampq_set_scale_mode(self._h, mode))
 
@@ -300,6 +306,12 @@ class Context:
 
     def last_launch_count(self) -> int:
         return lib().ampq_last_launch_count(self._h)
+
+    def get_pass_bytes(self) -> dict:
+        """Bytes of bound tensors the last pass reads: amax pass, scoring pass."""
+        b = (C.c_longlong * 2)()
+        self._check(lib().ampq_get_pass_bytes(self._h, b))
+        return dict(amax=int(b[0]), score=int(b[1]))
 
     def set_timing(self, on: bool):
         self._check(lib().ampq_set_timing(self._h, 1 if on else 0))

@@ -51,11 +51,23 @@ struct Tensor {
     int R;                   // calibration samples
     int per_sample;          // 1: values are [R, seg_len]; 0: shared by all samples
     int dtype;               // AMPQ_F32 / AMPQ_BF16
-    int rgroups;             // unused by the kernels (kept for table dumps): ceil(R / kMaxRB) or 1
+    int share_n;             // layers that read one per-sample operand are scored in one read of its values:
+                             // 1: on its own; n = 2..kMaxRB: first of n such tensors, its tiles carry the
+                             // gradient streams of all n; 0: one of the others (no tiles of its own)
     int seg_base;            // index of segment (this tensor, r = 0) in the segment outputs
     float amax_preset;       // >= 0: use instead of measuring
     int causal_shift;        // > 0: segments are stacks of T x T matrices, T = 2^causal_shift, whose strictly
                              // upper triangles are exactly zero and are not read; 0: dense
+    int amax_src;            // index of the tensor whose measured amax this one takes (a tensor bound to the
+                             // very same values); its own index otherwise
+    // Gradient streams 1..kMaxRB-1 of a tile that reads its values once for several
+    // streams (stream 0 is `grads`); stream j of a tile at sample r0 starts at
+    // gstream[j-1] + r0*grad_stride.  Shared values (weights): grads + j*grad_stride,
+    // the next samples' gradients.  share_n > 1: the gradients of tensors
+    // 1..share_n-1 of the group.  stream_slot_stride = partial slots between two
+    // streams: tiles_per_seg (next sample) or R*tiles_per_seg (next tensor).
+    const void* gstream[kMaxRB - 1];
+    long long stream_slot_stride;
 };
 
 // One segment = (tensor, sample): its partial slots are contiguous.

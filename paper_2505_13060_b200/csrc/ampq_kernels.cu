@@ -20,6 +20,7 @@
 //   codes_kernel    test hook: the FP8 codes the scoring kernel sees
 #include <cuda_runtime.h>
 #include <cuda_fp16.h>
+#include <atomic>
 #include <cstdint>
 
 #include "ampq_device.h"
@@ -138,6 +139,14 @@ __global__ void init_amax_kernel(const Tensor* __restrict__ tens, int T,
     }
 }
 
+// The alias step of scales_kernel alone, for passes that stop after the amax.
+__global__ void resolve_amax_kernel(int T, const Tensor* __restrict__ tens, unsigned* __restrict__ amax_bits) {
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const int src = tens[t].amax_src;
+    if (src != t) amax_bits[t] = amax_bits[src];
+}
+
 __global__ void __launch_bounds__(kThreads)
 amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
             unsigned* __restrict__ amax_bits) {
@@ -253,12 +262,18 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
 // 1/p.  With fmax = 1.75 * 2^ef and amax = m * 2^ea (1 <= m < 2) that is
 // 2^(ea - ef) when m <= 1.75 and 2^(ea - ef + 1) otherwise, read off the bits;
 // neutral when p or 1/p is not a normal fp32.
-__global__ void scales_kernel(int T, int fmask, const unsigned* __restrict__ amax_bits,
+//
+// A tensor bound to the same values as an earlier one (Tensor::amax_src) takes
+// that tensor's amax and records it as its own; the source always holds its own
+// amax, so no thread reads a word another one writes.
+__global__ void scales_kernel(int T, int fmask, const Tensor* __restrict__ tens, unsigned* __restrict__ amax_bits,
                               float* __restrict__ scales, int* __restrict__ tensor_flags,
                               LaunchStatus* status, int pow2) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
-    unsigned bits = amax_bits[t];
+    const int src = tens[t].amax_src;
+    unsigned bits = amax_bits[src];
+    if (src != t) amax_bits[t] = bits;
     int bad = bits >= 0x7F800000u;
     tensor_flags[t] = bad;
     if (bad) atomicExch(&status->nonfinite, 1);
@@ -661,7 +676,7 @@ template <int RB, bool CAUSAL>
 __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, int tile_shift) {
     TileGeom q;
     int i;  // value tile within the segment
-    if (tn.per_sample) {  // RB == 1
+    if (tn.per_sample) {  // one sample per tile; RB > 1: the RB streams are RB layers' gradients of that sample
         q.r0 = local / tn.tiles_per_seg;
         i = local - q.r0 * tn.tiles_per_seg;
         q.voff = (long long)q.r0 * tn.seg_len + ((long long)i << tile_shift);
@@ -695,6 +710,17 @@ __device__ __forceinline__ TileGeom tile_geometry(const Tensor& tn, int local, i
     return q;
 }
 
+// Gradient streams of a tile (Tensor::gstream): the next samples of a shared
+// operand's own gradients, or the gradients of the other layers that read this
+// per-sample operand.
+template <int RB, int ES>
+__device__ __forceinline__ void grad_bases(const Tensor& tn, const TileGeom& q, const char* (&gb)[RB]) {
+    const long long off = (q.goff + (long long)q.r0 * tn.grad_stride) * ES;
+    gb[0] = reinterpret_cast<const char*>(tn.grads) + off;
+#pragma unroll
+    for (int r = 1; r < RB; ++r) gb[r] = reinterpret_cast<const char*>(tn.gstream[r - 1]) + off;
+}
+
 // Debug builds (-DAMPQ_BOUNDS_CHECK): a tile whose element range, samples or
 // partial slots fall outside what its tensor owns is reported in the status
 // word and skipped by the producer and the scoring warps alike, instead of
@@ -704,9 +730,13 @@ template <int RB>
 __device__ __forceinline__ bool tile_in_bounds(const Tensor& tn, const TileGeom& q) {
 #ifdef AMPQ_BOUNDS_CHECK
     const long long vals = tn.per_sample ? tn.numel : tn.seg_len;
+    const long long per_tensor = (long long)tn.R * tn.tiles_per_seg;
+    const bool shared_input = RB > 1 && tn.per_sample;
+    const int last_r = shared_input ? q.r0 : q.r0 + RB - 1;
+    const long long owned = shared_input ? RB * per_tensor : per_tensor;
     return q.n > 0 && q.goff >= 0 && q.goff + q.n <= tn.seg_len && q.voff >= 0 && q.voff + q.n <= vals &&
-           q.r0 >= 0 && q.r0 + RB <= tn.R && q.slot0 >= tn.partial_base &&
-           q.slot0 + (long long)(RB - 1) * tn.tiles_per_seg < tn.partial_base + (long long)tn.R * tn.tiles_per_seg;
+           q.r0 >= 0 && last_r < tn.R && (!shared_input || tn.share_n == RB) && q.slot0 >= tn.partial_base &&
+           q.slot0 + (long long)(RB - 1) * tn.stream_slot_stride < tn.partial_base + owned;
 #else
     return true;
 #endif
@@ -763,12 +793,10 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
                 constexpr int es = Elem<DT>::kBytes;
                 const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
                 const char* gb[RB];
+                grad_bases<RB, es>(tn, q, gb);
                 bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
 #pragma unroll
-                for (int r = 0; r < RB; ++r) {
-                    gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
-                    aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
-                }
+                for (int r = 0; r < RB; ++r) aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
                 const int nchunks = aligned && tile_in_bounds<RB>(tn, q) ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
                 for (int c = 0; c < nchunks; ++c) {
                     // the stage must have been handed back once per earlier lap
@@ -817,12 +845,10 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         }
         const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
         const char* gb[RB];
+        grad_bases<RB, es>(tn, q, gb);
         bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
 #pragma unroll
-        for (int r = 0; r < RB; ++r) {
-            gb[r] = reinterpret_cast<const char*>(tn.grads) + (q.goff + (long long)(q.r0 + r) * tn.grad_stride) * es;
-            aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
-        }
+        for (int r = 0; r < RB; ++r) aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
         const bool inside = tile_in_bounds<RB>(tn, q);
         if (!inside) {  // only in a bounds-checking build: report, score nothing, move on
             if (threadIdx.x == 0) atomicExch(&status->bounds, 1);
@@ -852,7 +878,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
             score_direct<DT, FMASK, RB>(vb + (long long)done * es, gt, q.n - done, inv2, nsc2, acc64);
         }
         reduce_and_store<NACC, RB>(acc64, s_red + red_block * (kConsumers / 32) * RB * NACC, partials, q.slot0,
-                                   tn.tiles_per_seg, out_stride);
+                                   tn.stream_slot_stride, out_stride);
         red_block ^= 1;
     }
 }
@@ -949,10 +975,13 @@ __global__ void job_prepare_kernel(SegmentJob* job, const void* values, const vo
     t.R = 1;
     t.per_sample = 1;
     t.dtype = dtype;
-    t.rgroups = 1;
+    t.share_n = 1;
     t.seg_base = 0;
     t.amax_preset = amax_preset;
     t.causal_shift = 0;
+    t.amax_src = 0;
+    for (int k = 0; k < kMaxRB - 1; ++k) t.gstream[k] = nullptr;
+    t.stream_slot_stride = ntiles;
     job->tensor = t;
     job->tile_begin[0] = 0;
     job->tile_begin[1] = ntiles;
@@ -1020,10 +1049,16 @@ cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
+cudaError_t launch_scales(int T, int fmask, const Tensor* tens, unsigned* amax_bits, float* scales, int* tensor_flags,
                           LaunchStatus* status, cudaStream_t st, int pow2) {
     if (T <= 0) return cudaSuccess;
-    scales_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, fmask, amax_bits, scales, tensor_flags, status, pow2);
+    scales_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, fmask, tens, amax_bits, scales, tensor_flags, status, pow2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_resolve_amax(int T, const Tensor* tens, unsigned* amax_bits, cudaStream_t st) {
+    if (T <= 0) return cudaSuccess;
+    resolve_amax_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, tens, amax_bits);
     return cudaGetLastError();
 }
 
@@ -1039,9 +1074,16 @@ static cudaError_t launch_score_inst(const Tensor* tens, const long long* tile_b
                                      LaunchStatus* status, cudaStream_t st, int out_stride) {
     constexpr int smem = Ring<RB>::kSmemBytes;
     if (out_stride < Fm<FMASK>::kAcc) out_stride = Fm<FMASK>::kAcc;
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB, CAUSAL>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    // the shared-memory opt-in of an instantiation is set once per device
+    static std::atomic<unsigned long long> opted_in{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev >= 64 || !(opted_in.load(std::memory_order_acquire) >> dev & 1ULL)) {
+        e = cudaFuncSetAttribute(score_kernel<DT, FMASK, RB, CAUSAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev < 64) opted_in.fetch_or(1ULL << dev, std::memory_order_release);
+    }
     const unsigned grid = (unsigned)(ntiles < (long long)max_ctas ? ntiles : (long long)max_ctas);
     score_kernel<DT, FMASK, RB, CAUSAL><<<grid, kScoreThreads, smem, st>>>(tens, tile_begin, T, ntiles, tile_shift,
                                                                            scales, partials, status, out_stride);

@@ -18,11 +18,15 @@ cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, Lau
                              cudaStream_t st);
 cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
                         unsigned* amax_bits, cudaStream_t st);
-// pow2 = 1: power-of-two scales instead of amax / fmax.
-cudaError_t launch_scales(int T, int fmask, const unsigned* amax_bits, float* scales, int* tensor_flags,
+// pow2 = 1: power-of-two scales instead of amax / fmax.  Tensors whose amax_src
+// names another tensor take (and record) that tensor's amax.
+cudaError_t launch_scales(int T, int fmask, const Tensor* tens, unsigned* amax_bits, float* scales, int* tensor_flags,
                           LaunchStatus* status, cudaStream_t st, int pow2 = 0);
-// One launch per element type (0 = fp32, 1 = bf16) and sample-group size rb =
-// 1..kMaxRB, each with its own tile table; causal = 1 (rb = 1 only): the
+// Only that alias step (after an amax pass that is not followed by a score).
+cudaError_t launch_resolve_amax(int T, const Tensor* tens, unsigned* amax_bits, cudaStream_t st);
+// One launch per element type (0 = fp32, 1 = bf16) and number of gradient
+// streams per read of the values rb = 1..kMaxRB (samples of a shared operand, or
+// layers reading one per-sample operand), each with its own tile table; causal = 1 (rb = 1 only): the
 // table holds triangular operands (Tensor::causal_shift > 0).  fmask = 0 scores
 // only S (no cast, scales unused).  out_stride = doubles per partial slot when
 // that is more than the kernel's own accumulator count (0: exactly that count).

@@ -111,6 +111,7 @@ struct ampq_ctx {
     std::vector<Group> groups;
     int scale_pow2 = 0;    // AMPQ_SCALE_POW2: power-of-two scales
     bool measured = true;  // false: only the model term S is scored (no amax pass, no cast)
+    bool sharing = true;   // layers bound to the very same values share its amax and one read of it
     bool amax_ready = false;  // ampq_measure_amax (or a score) has filled the amax mirror
     bool dirty = true;     // bindings changed since the tables were built
     bool scored = false;   // a score has been issued
@@ -128,7 +129,9 @@ struct ampq_ctx {
     std::vector<Layer> lay;
     std::vector<int> scored_layer_ids;
     long long ntiles[kScoreClasses] = {}, namax_tiles = 0, nslots = 0;
-    std::vector<std::pair<int, int>> amax_alias;  // (tensor, earlier tensor bound to the very same values)
+    int n_amax_alias = 0;     // tensors that take an earlier tensor's amax (bound to the very same values)
+    int n_share_groups = 0;   // groups of layers scored in one read of a per-sample operand they share
+    long long amax_bytes = 0, score_bytes = 0;  // bytes of bound tensors the two passes of a score read
     int layer_out_doubles = 0;
 
     DevBuf<Tensor> d_tens;
@@ -244,20 +247,72 @@ int causal_shift_of(const LayerRec& l, const Operand& o, const Tensor& t) {
     return shift;
 }
 
+// What makes two per-sample operands "the same input read by several layers".
+struct ShareKey {
+    const void* values;
+    long long numel, grad_stride;
+    int dtype, R;
+    unsigned preset_bits;
+    bool operator==(const ShareKey& o) const {
+        return values == o.values && numel == o.numel && grad_stride == o.grad_stride && dtype == o.dtype && R == o.R &&
+               preset_bits == o.preset_bits;
+    }
+};
+
+struct ShareGroup {
+    ShareKey key;
+    std::vector<const Operand*> members;  // in registration order; members[0] carries the tiles
+    int leader_tensor = -1;
+    long long leader_base = 0;
+    int leader_amax_src = -1;
+};
+
 // Builds the host tables for every layer whose two operands are bound.
 int build_tables(ampq_ctx* ctx) {
-    ctx->tens.clear(); ctx->amax_tile_begin.clear(); ctx->amax_alias.clear();
+    ctx->tens.clear(); ctx->amax_tile_begin.clear();
+    ctx->n_amax_alias = 0; ctx->n_share_groups = 0;
+    ctx->amax_bytes = 0; ctx->score_bytes = 0;
     for (auto& tb : ctx->tile_begin) tb.clear();
     ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
     for (auto& l : ctx->layers) { l.scored = -1; l.op[0].tensor = l.op[1].tensor = -1; }
     long long tiles[kScoreClasses] = {}, atiles = 0, slots = 0;
     int out_off = 0;
     std::vector<char> measures_amax;  // per tensor: it has amax tiles of its own
+
+    // Layers that read one input (q, k, v or gate, up of a transformer block) bind
+    // the very same per-sample values with gradients of their own.  Up to kMaxRB
+    // of them form a group that is scored like a weight with several per-sample
+    // gradients: the values are read and cast once per tile, every member's
+    // gradient is one more stream of that tile.
+    std::vector<ShareGroup> groups;
+    std::vector<std::pair<int, int>> role(ctx->layers.size() * 2, {-1, 0});  // (group, position) per operand
+    if (ctx->sharing) {
+        for (size_t li = 0; li < ctx->layers.size(); ++li) {
+            const LayerRec& l = ctx->layers[li];
+            if (!layer_ready(l)) continue;
+            for (int k = 0; k < 2; ++k) {
+                const Operand& o = l.op[k];
+                if (o.mem != AMPQ_MEM_DEVICE || !o.per_sample || o.numel == 0 || o.causal_T != 0) continue;
+                unsigned pb;
+                std::memcpy(&pb, &o.amax_preset, sizeof pb);
+                const ShareKey key{o.values, o.numel, o.grad_stride, o.dtype, l.R, pb};
+                int g = -1;
+                for (size_t e = groups.size(); e-- > 0;)  // the latest group of this key that still has room
+                    if (groups[e].key == key) { if ((int)groups[e].members.size() < kMaxRB) g = (int)e; break; }
+                if (g < 0) { groups.push_back(ShareGroup{key, {}, -1, 0, -1}); g = (int)groups.size() - 1; }
+                role[2 * li + k] = {g, (int)groups[g].members.size()};
+                groups[g].members.push_back(&o);
+            }
+        }
+    }
     long long scored_elems = 0;  // value elements the scoring launches walk (shared values once per sample group)
-    for (const auto& l : ctx->layers) {
+    for (size_t li = 0; li < ctx->layers.size(); ++li) {
+        const LayerRec& l = ctx->layers[li];
         if (!layer_ready(l)) continue;
-        for (int k = 0; k < 2; ++k)
+        for (int k = 0; k < 2; ++k) {
+            if (role[2 * li + k].first >= 0 && role[2 * li + k].second > 0) continue;  // read with its group's first member
             scored_elems += l.op[k].per_sample ? l.op[k].numel : l.op[k].numel * ((l.R + kMaxRB - 1) / kMaxRB);
+        }
     }
     ctx->tile_shift = pick_tile_shift(scored_elems, ctx->max_ctas);
     const long long tile_elems = 1LL << ctx->tile_shift;
@@ -301,37 +356,80 @@ int build_tables(ampq_ctx* ctx) {
             if ((ext + tile_elems - 1) / tile_elems > 0x7FFFFFFFLL)
                 return fail(ctx, AMPQ_ERR_TOO_LARGE, "an operand has more than 2^31-1 tiles per sample");
             t.tiles_per_seg = (int)((ext + tile_elems - 1) / tile_elems);
-            t.rgroups = o.per_sample ? 1 : (l.R + kMaxRB - 1) / kMaxRB;
-            t.partial_base = slots;
+            t.share_n = 1;
+            t.stream_slot_stride = t.tiles_per_seg;
+            for (int j = 1; j < kMaxRB; ++j)  // never read past the R samples: a tile of a shared operand has at most R streams
+                t.gstream[j - 1] = reinterpret_cast<const char*>(t.grads) + (long long)j * t.grad_stride * es;
             t.seg_base = (int)ctx->segs.size();
             t.amax_preset = o.amax_preset;
             t.causal_shift = causal_shift_of(l, o, t);
+            const int me = (int)ctx->tens.size();
+            t.amax_src = me;
+            const long long per_tensor_slots = (long long)l.R * t.tiles_per_seg;
+            ShareGroup* grp = role[2 * li + k].first >= 0 ? &groups[role[2 * li + k].first] : nullptr;
+            const int pos = role[2 * li + k].second;
+            if (grp && grp->members.size() < 2) grp = nullptr;
             // per-sample operands: one single-sample tile per (sample, value tile);
             // shared operands: value tiles x full groups of kMaxRB samples, plus one
-            // remainder group of R mod kMaxRB samples
+            // remainder group of R mod kMaxRB samples; an input read by n layers: the
+            // first layer's tensor has one n-stream tile per (sample, value tile)
             long long my_tiles[kScoreClasses] = {};
             const int c0 = (o.dtype == AMPQ_F32 ? 0 : 1) * kMaxRB;  // classes of this operand's dtype
-            if (t.causal_shift > 0) {
-                my_tiles[2 * kMaxRB + (o.dtype == AMPQ_F32 ? 0 : 1)] = (long long)l.R * t.tiles_per_seg;
-            } else if (o.per_sample) {
-                my_tiles[c0] = (long long)l.R * t.tiles_per_seg;
-            } else {
-                my_tiles[c0 + kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
-                if (l.R % kMaxRB) my_tiles[c0 + l.R % kMaxRB - 1] += t.tiles_per_seg;
-            }
             long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
-            // Layers that read the same tensor (q, k, v or gate, up of one block share
-            // their input) need its amax only once: a later binding of the very same
-            // device values takes the amax of the first instead of another read.
-            if (my_atiles > 0 && o.mem == AMPQ_MEM_DEVICE) {
-                for (size_t e = 0; e < ctx->tens.size(); ++e) {
-                    const Tensor& u = ctx->tens[e];
-                    if (measures_amax[e] && u.values == t.values && u.numel == t.numel && u.dtype == t.dtype &&
-                        u.causal_shift == t.causal_shift) {
-                        ctx->amax_alias.emplace_back((int)ctx->tens.size(), (int)e);
-                        my_atiles = 0;
-                        break;
+            if (grp && pos > 0) {
+                t.share_n = 0;
+                t.partial_base = grp->leader_base + pos * per_tensor_slots;
+                if (my_atiles > 0) { t.amax_src = grp->leader_amax_src; ++ctx->n_amax_alias; }
+                my_atiles = 0;
+            } else {
+                t.partial_base = slots;
+                if (grp) {
+                    const int n = (int)grp->members.size();
+                    t.share_n = n;
+                    for (int j = 1; j < n; ++j) t.gstream[j - 1] = grp->members[j]->grads;
+                    t.stream_slot_stride = per_tensor_slots;
+                    my_tiles[c0 + n - 1] = per_tensor_slots;
+                    grp->leader_tensor = me;
+                    grp->leader_base = slots;
+                    slots += (long long)n * per_tensor_slots;
+                    ++ctx->n_share_groups;
+                } else {
+                    if (t.causal_shift > 0) my_tiles[2 * kMaxRB + (o.dtype == AMPQ_F32 ? 0 : 1)] = per_tensor_slots;
+                    else if (o.per_sample) my_tiles[c0] = per_tensor_slots;
+                    else {
+                        my_tiles[c0 + kMaxRB - 1] = (long long)t.tiles_per_seg * (l.R / kMaxRB);
+                        if (l.R % kMaxRB) my_tiles[c0 + l.R % kMaxRB - 1] += t.tiles_per_seg;
                     }
+                    slots += per_tensor_slots;
+                }
+                // A tensor bound to the very same device values as an earlier one needs no
+                // amax pass of its own: it takes the earlier one's.
+                if (ctx->sharing && my_atiles > 0 && o.mem == AMPQ_MEM_DEVICE) {
+                    for (size_t e = 0; e < ctx->tens.size(); ++e) {
+                        const Tensor& u = ctx->tens[e];
+                        if (measures_amax[e] && u.values == t.values && u.numel == t.numel && u.dtype == t.dtype &&
+                            u.causal_shift == t.causal_shift) {
+                            t.amax_src = (int)e;
+                            ++ctx->n_amax_alias;
+                            my_atiles = 0;
+                            break;
+                        }
+                    }
+                }
+                if (grp) grp->leader_amax_src = t.amax_src;
+            }
+            {
+                // bytes read: a triangular operand keeps, of row i, the 16-byte vectors up to the diagonal
+                long long kept = o.numel;
+                if (t.causal_shift > 0) {
+                    const long long T = 1LL << t.causal_shift, per = 16 / es, g = T / per;
+                    kept = o.numel / (T * T) * (per * per * g * (g + 1) / 2);
+                }
+                if (my_atiles > 0) ctx->amax_bytes += kept * es;
+                if (t.share_n > 0) {
+                    const long long value_reads = o.per_sample ? 1 : (l.R + kMaxRB - 1) / kMaxRB;
+                    const long long grad_streams = o.per_sample ? t.share_n : l.R;
+                    ctx->score_bytes += kept * es * (value_reads + grad_streams);
                 }
             }
             for (int c = 0; c < kScoreClasses; ++c) {
@@ -342,13 +440,12 @@ int build_tables(ampq_ctx* ctx) {
             atiles += my_atiles;
             measures_amax.push_back(my_atiles > 0);
             for (int r = 0; r < l.R; ++r) {
-                Segment s{};
-                s.first_slot = slots + (long long)r * t.tiles_per_seg;
-                s.count = t.tiles_per_seg;
-                ctx->segs.push_back(s);
+                Segment sg{};
+                sg.first_slot = t.partial_base + (long long)r * t.tiles_per_seg;
+                sg.count = t.tiles_per_seg;
+                ctx->segs.push_back(sg);
             }
-            slots += (long long)l.R * t.tiles_per_seg;
-            o.tensor = (int)ctx->tens.size();
+            o.tensor = me;
             if (k == 0) { ly.seg_base0 = t.seg_base; ly.tensor0 = o.tensor; }
             else { ly.seg_base1 = t.seg_base; ly.tensor1 = o.tensor; }
             ctx->tens.push_back(t);
@@ -492,14 +589,6 @@ int prepare_tables(ampq_ctx* ctx) {
     return AMPQ_OK;
 }
 
-// Tensors bound to the same values as an earlier one take that one's amax.
-int copy_alias_amax(ampq_ctx* ctx) {
-    for (const auto& a : ctx->amax_alias)
-        AMPQ_CUDA(cudaMemcpyAsync(ctx->d_amax_bits.p + a.first, ctx->d_amax_bits.p + a.second, sizeof(unsigned),
-                                  cudaMemcpyDeviceToDevice, ctx->stream), "D2D amax");
-    return AMPQ_OK;
-}
-
 // Per-layer combine and the asynchronous read-back of every small result.
 int combine_and_read_back(ampq_ctx* ctx, int T, int L, int S) {
     const int nacc = ctx->F;
@@ -526,7 +615,7 @@ int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, LaunchStatus* status, in
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
     AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, st), "job_prepare");
     AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st), "amax");
-    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->amax_bits, job->scales, &job->flag, status, st, ctx->scale_pow2), "scales");
+    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->tensor, &job->amax_bits, job->scales, &job->flag, status, st, ctx->scale_pow2), "scales");
     return AMPQ_OK;
 }
 
@@ -599,6 +688,7 @@ int ampq_set_formats(ampq_ctx* ctx, const int* fmt, int F) {
     if (!ctx || !fmt) return AMPQ_ERR_INVALID;
     if (F < 2 || F > 1 + kMaxLow) return fail(ctx, AMPQ_ERR_INVALID, "F must be 2 or 3");
     if (fmt[0] != AMPQ_FMT_BASE) return fail(ctx, AMPQ_ERR_INVALID, "fmt[0] must be AMPQ_FMT_BASE");
+    if (ctx->streaming) return fail(ctx, AMPQ_ERR_STATE, "the formats cannot change inside a streaming pass");
     int mask = 0;
     for (int f = 1; f < F; ++f) {
         if (fmt[f] != AMPQ_FMT_E4M3 && fmt[f] != AMPQ_FMT_E5M2) return fail(ctx, AMPQ_ERR_INVALID, "unknown low-precision format");
@@ -657,7 +747,7 @@ int ampq_set_amax(ampq_ctx* ctx, int layer_id, int operand, float amax) {
     if (rc) return rc;
     if (operand != 0 && operand != 1) return fail(ctx, AMPQ_ERR_INVALID, "operand must be 0 or 1");
     if (amax != amax || std::isinf(amax)) return fail(ctx, AMPQ_ERR_INVALID, "amax must be finite");
-    ctx->layers[layer_id].op[operand].amax_preset = amax >= 0.0f ? amax : -1.0f;
+    ctx->layers[layer_id].op[operand].amax_preset = amax > 0.0f ? amax : (amax == 0.0f ? 0.0f : -1.0f);  // -0 -> +0
     ctx->dirty = true;
     return AMPQ_OK;
 }
@@ -665,6 +755,7 @@ int ampq_set_amax(ampq_ctx* ctx, int layer_id, int operand, float amax) {
 int ampq_set_scale_mode(ampq_ctx* ctx, int mode) {
     if (!ctx) return AMPQ_ERR_INVALID;
     if (mode != AMPQ_SCALE_AMAX && mode != AMPQ_SCALE_POW2) return fail(ctx, AMPQ_ERR_INVALID, "unknown scale mode");
+    if (ctx->streaming) return fail(ctx, AMPQ_ERR_STATE, "the scale mode cannot change inside a streaming pass");
     ctx->scale_pow2 = mode == AMPQ_SCALE_POW2 ? 1 : 0;
     ctx->scored = false;
     return AMPQ_OK;
@@ -672,8 +763,16 @@ int ampq_set_scale_mode(ampq_ctx* ctx, int mode) {
 
 int ampq_set_measured(ampq_ctx* ctx, int on) {
     if (!ctx) return AMPQ_ERR_INVALID;
+    if (ctx->streaming) return fail(ctx, AMPQ_ERR_STATE, "the scored terms cannot change inside a streaming pass");
     ctx->measured = on != 0;
     ctx->scored = false;
+    return AMPQ_OK;
+}
+
+int ampq_set_sharing(ampq_ctx* ctx, int on) {
+    if (!ctx) return AMPQ_ERR_INVALID;
+    ctx->sharing = on != 0;
+    ctx->dirty = true;
     return AMPQ_OK;
 }
 
@@ -693,7 +792,10 @@ int ampq_measure_amax(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
         AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
         ctx->launches = ctx->namax_tiles > 0 ? 2 : 1;
-        if ((rc = copy_alias_amax(ctx))) return rc;
+        if (ctx->n_amax_alias > 0) {
+            AMPQ_CUDA(launch_resolve_amax(T, ctx->d_tens.p, ctx->d_amax_bits.p, st), "resolve_amax");
+            ++ctx->launches;
+        }
         AMPQ_CUDA(cudaMemcpyAsync(ctx->h_amax_bits.p, ctx->d_amax_bits.p, T * sizeof(unsigned), cudaMemcpyDeviceToHost, st), "D2H amax");
     }
     ctx->amax_ready = true;
@@ -748,12 +850,11 @@ int ampq_score(ampq_ctx* ctx) {
         if (ctx->namax_tiles > 0 && ctx->measured) {
             AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
             ++ctx->launches;
-            if ((rc = copy_alias_amax(ctx))) return rc;
         }
         if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched
             AMPQ_CUDA(cudaMemsetAsync(ctx->d_partials.p, 0, (size_t)ctx->nslots * nacc * sizeof(double), st), "memset partials");
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
-        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
+        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         for (int c = 0; c < kScoreClasses; ++c) {
@@ -907,7 +1008,7 @@ int ampq_fake_quant(ampq_ctx* ctx, int dtype, int fmt, const void* values, long 
     AMPQ_CUDA(ctx->d_fq_job.ensure(1), "cudaMalloc(job)");
     AMPQ_CUDA(ctx->d_fq_status.ensure(1), "cudaMalloc(status)");
     int rc = job_amax_and_scales(ctx, ctx->d_fq_job.p, ctx->d_fq_status.p, dtype, values, values, numel,
-                                 amax >= 0.0f ? amax : -1.0f, 0);
+                                 amax > 0.0f ? amax : (amax == 0.0f ? 0.0f : -1.0f), 0);
     if (rc) return rc;
     const float* pair = ctx->d_fq_job.p->scales + ctx->slot_of_fmt[f] * 2;
     AMPQ_CUDA(launch_fake_quant(dtype, fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2, values, numel, pair, dev_out, ctx->stream), "fake_quant");
@@ -915,6 +1016,15 @@ int ampq_fake_quant(ampq_ctx* ctx, int dtype, int fmt, const void* values, long 
 }
 
 int ampq_last_launch_count(const ampq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int ampq_get_pass_bytes(ampq_ctx* ctx, long long* bytes) {
+    if (!ctx || !bytes) return AMPQ_ERR_INVALID;
+    if (ctx->dirty || ctx->streaming || !(ctx->scored || ctx->amax_ready))
+        return fail(ctx, AMPQ_ERR_STATE, "no pass has been issued for the current bindings");
+    bytes[0] = ctx->measured ? ctx->amax_bytes : 0;
+    bytes[1] = ctx->score_bytes;
+    return AMPQ_OK;
+}
 
 int ampq_set_timing(ampq_ctx* ctx, int on) {
     if (!ctx) return AMPQ_ERR_INVALID;

@@ -70,10 +70,13 @@ __global__ void noalloc_prepare_kernel(NoAllocScratch* s, const void* values, co
     t.R = 1;
     t.per_sample = 1;
     t.dtype = dtype;
-    t.rgroups = 1;
+    t.share_n = 1;
     t.seg_base = 0;
     t.amax_preset = amax_preset;
     t.causal_shift = 0;
+    t.amax_src = 0;
+    for (int k = 0; k < kMaxRB - 1; ++k) t.gstream[k] = nullptr;
+    t.stream_slot_stride = ntiles;
     s->tensor = t;
     s->tile_begin[0] = 0;
     s->tile_begin[1] = ntiles;
@@ -151,7 +154,7 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     if (scratch_of(device, &s) != cudaSuccess) { cudaGetLastError(); return AMPQ_ERR_CUDA; }
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-    const float preset = amax >= 0.0f ? amax : -1.0f;
+    const float preset = amax > 0.0f ? amax : (amax == 0.0f ? 0.0f : -1.0f);  // -0 -> +0
     const long long ntiles = (numel + kTileElems - 1) / kTileElems;
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
     const int fmask = fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2;
@@ -159,7 +162,7 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     bool ok = cudaGetLastError() == cudaSuccess;
     ok = ok && launch_init_amax(&s->tensor, 1, &s->amax_bits, &s->status, st) == cudaSuccess;
     ok = ok && launch_amax(&s->tensor, s->amax_tile_begin, 1, namax, &s->amax_bits, st) == cudaSuccess;
-    ok = ok && launch_scales(1, fmask, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
+    ok = ok && launch_scales(1, fmask, &s->tensor, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
     int sms = 0;
     ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
     ok = ok && launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &s->tensor, s->tile_begin, 1, ntiles, kMaxTileShift, kScoreCtasPerSm * sms, fmask, s->scales,

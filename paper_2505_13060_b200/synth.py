@@ -184,6 +184,19 @@ def make_layer(spec: LayerSpec, device, seed: int = 0, layer: int = 0) -> LayerT
     return lt
 
 
+def share_block_inputs(lts: list) -> None:
+    """Makes the layers of one transformer block that read the same activation
+    bind the same tensor, as they do in a model: k and v take q's input, up takes
+    gate's.  Every layer keeps the gradient with respect to its own input."""
+    by_name = {lt.spec.name.split(".")[-1]: lt for lt in lts}
+    for first, others in (("q", ("k", "v")), ("gate", ("up",))):
+        if first not in by_name:
+            continue
+        for o in others:
+            if o in by_name and by_name[o].values[0].shape == by_name[first].values[0].shape:
+                by_name[o].values[0] = by_name[first].values[0]
+
+
 def to_numpy(t: torch.Tensor):
     """Host copy for the oracle: fp32 as float32, bf16 as its uint16 bit pattern."""
     t = t.detach().contiguous().cpu()

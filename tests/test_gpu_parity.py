@@ -580,3 +580,78 @@ def test_layers_sharing_one_input_tensor(ampq, orc):
     compare_layer(ampq, ctx, ids[1], oracle_layer(orc, lts[1], [E4M3], amax_presets=(2.0, None)), 2, "preset sibling")
     compare_layer(ampq, ctx, ids[2], refs[2], 2, "unpreset sibling")
     ctx.destroy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("members", [2, 3, 4, 5, 9])
+def test_shared_input_groups_score_in_one_read(ampq, orc, dtype, members):
+    """`members` layers bind one per-sample input (their own gradients and
+    weights): up to four at a time are scored in one read of the values, the
+    rest in further groups.  Every layer's values equal the oracle's and, bit
+    for bit in amax and scales, those of the same layers scored one by one
+    (sharing off); the pass reads the shared input once per group.  Ragged
+    sizes, a gradient that is not 16-byte aligned, another stride and another R
+    (which must not join a group) are mixed in."""
+    R, n = 3, 70001 if dtype == torch.float32 else 140011
+    es = torch.empty((), dtype=dtype).element_size()
+    g = torch.Generator(device="cuda").manual_seed(17 + members)
+    X = torch.empty(R * n, dtype=dtype, device="cuda").normal_(0, 1, generator=g)
+
+    class LT:
+        pass
+
+    lts = []
+    for m in range(members):
+        lt = LT()
+        lt.spec = synth.LayerSpec("m%d" % m, synth.LINEAR, R, dtype, synth.OperandSpec((R, n), True),
+                                  synth.OperandSpec((300 + m,), False))
+        off = 1 if m == 2 else 0   # one member's gradient starts one element past a 16-byte boundary
+        gbuf = torch.empty(R * n + 8, dtype=dtype, device="cuda").normal_(0, 1e-3, generator=g)
+        lt.values = [X, torch.empty(300 + m, dtype=dtype, device="cuda").normal_(0, 0.02, generator=g)]
+        lt.grads = [gbuf[off:off + R * n], torch.empty(R, 300 + m, dtype=dtype, device="cuda").normal_(0, 1e-3, generator=g)]
+        lts.append(lt)
+
+    def bind(ctx):
+        ids = []
+        for lt in lts:
+            lid = ctx.register_layer(ampq.LINEAR, lt.spec.name, R)
+            code = ampq.torch_dtype_code(X)
+            ctx.bind_operand(lid, 0, code, X.data_ptr(), R * n, True, lt.grads[0].data_ptr(), n)
+            ctx.bind_operand(lid, 1, code, lt.values[1].data_ptr(), lt.values[1].numel(), False,
+                             lt.grads[1].data_ptr(), lt.values[1].numel())
+            ids.append(lid)
+        return ids
+
+    shared = _ctx(ampq, (0, E4M3, E5M2))
+    ids = bind(shared)
+    # the same X with a larger gradient stride, and its first two samples as an R = 2 layer: never grouped
+    wide = torch.empty(R * (n + 5), dtype=dtype, device="cuda").normal_(0, 1e-3, generator=g)
+    odd = shared.register_layer(ampq.LINEAR, "stride", R)
+    shared.bind_operand(odd, 0, ampq.torch_dtype_code(X), X.data_ptr(), R * n, True, wide.data_ptr(), n + 5)
+    shared.bind_operand(odd, 1, ampq.torch_dtype_code(X), lts[0].values[1].data_ptr(), 300, False, lts[0].grads[1].data_ptr(), 300)
+    shared.score()
+    alone = _ctx(ampq, (0, E4M3, E5M2))
+    alone.set_sharing(False)
+    ids2 = bind(alone)
+    alone.score()
+    refs = [oracle_layer(orc, lt, [E4M3, E5M2]) for lt in lts]
+    for lid, lid2, lt, ref in zip(ids, ids2, lts, refs):
+        got = compare_layer(ampq, shared, lid, ref, 3, "group member " + lt.spec.name)
+        sep = compare_layer(ampq, alone, lid2, ref, 3, "scored alone " + lt.spec.name)
+        assert got["amax"].tobytes() == sep["amax"].tobytes() and got["scale"].tobytes() == sep["scale"].tobytes()
+        assert_close(got["s_per_sample"], sep["s_per_sample"], "group vs alone", 1e-9)
+        want = orc.codes(synth.to_numpy(X), E4M3, ref["ops"][0]["inv"][0])
+        assert np.array_equal(gpu_codes(shared, lid, 0, E4M3, X.numel()), want)
+    wide_ref = orc.score_operand(synth.to_numpy(X).reshape(R, -1),
+                                 synth.to_numpy(wide).reshape(R, n + 5)[:, :n].copy(), R, True, [E4M3, E5M2])
+    assert_close(shared.get_operand(odd, 0), wide_ref[3], "member with another gradient stride")
+    # bytes read: X once per group of up to four (plus the odd one) against once per layer
+    groups = (members + 3) // 4
+    xb = R * n * es
+    wb = sum(lt.values[1].numel() for lt in lts) * es
+    assert shared.get_pass_bytes()["amax"] == xb + wb   # the extra layer's two operands alias X and the first weight
+    assert alone.get_pass_bytes()["amax"] == members * xb + wb
+    assert shared.get_pass_bytes()["score"] == (groups + members) * xb + 2 * xb + wb * (1 + R) + 300 * es * (1 + R)
+    assert alone.get_pass_bytes()["score"] == 2 * members * xb + wb * (1 + R)
+    shared.destroy()
+    alone.destroy()
