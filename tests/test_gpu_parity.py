@@ -639,7 +639,7 @@ def test_shared_input_groups_score_in_one_read(ampq, orc, dtype, members):
         got = compare_layer(ampq, shared, lid, ref, 3, "group member " + lt.spec.name)
         sep = compare_layer(ampq, alone, lid2, ref, 3, "scored alone " + lt.spec.name)
         assert got["amax"].tobytes() == sep["amax"].tobytes() and got["scale"].tobytes() == sep["scale"].tobytes()
-        assert_close(got["s_per_sample"], sep["s_per_sample"], "group vs alone", 1e-9)
+        assert_close(got["s_per_sample"], sep["s_per_sample"], "group vs alone", 2e-6)  # other fp32 run lengths
         want = orc.codes(synth.to_numpy(X), E4M3, ref["ops"][0]["inv"][0])
         assert np.array_equal(gpu_codes(shared, lid, 0, E4M3, X.numel()), want)
     wide_ref = orc.score_operand(synth.to_numpy(X).reshape(R, -1),
