@@ -21,7 +21,8 @@
  *     last equation) -> orc_group_costs;
  *   - the integer program of Sec. 2.1 (maximise sum c subject to sum d <=
  *     budget, one configuration per group) -> orc_select_bruteforce,
- *     orc_select_bnb;
+ *     orc_select_bnb (plain depth-first search), orc_select_dp_integer (the
+ *     textbook dynamic program, for integer-valued d);
  *   - budget tau^2 E[g^2] (Sec. 2.1; E[g^2] is the mean-square loss of
  *     Algorithm 1 step 2) -> orc_budget_from_tau.
  *   - The paper only models the quantisation error; the measured error term
@@ -382,44 +383,31 @@ int orc_select_bruteforce(int J, const int *P, const long long *off, const doubl
     return 0;
 }
 
-/* Depth-first branch and bound for problems too large to enumerate.  Explores
- * assignments in lexicographic order with exactly the same left-fold sums as
- * the enumeration; a sub-tree is cut only when (a) even its smallest possible
- * d exceeds the budget, or (b) an upper bound on its c (the linear relaxation
- * of the remaining multiple-choice knapsack: per group the upper convex hull of
- * its (d, c) points, increments taken greedily by slope) is below the incumbent
- * by more than a rounding margin.  Cuts never use equality, so ties are still
- * resolved by the ordering above. */
-typedef struct { double dd, dc, slope; int j, to; } orc_seg;
-
+/* Depth-first branch and bound for problems too large to enumerate (Sec. 2.1,
+ * the integer program).  Groups are taken in order j = 0..J-1 and configurations
+ * in order p = 0..P_j-1, so leaves are met in lexicographic order and carry
+ * exactly the left-fold sums of the enumeration.  Below a node with partial
+ * sums (cs, ds) over groups < j, a leaf's sums are those partial sums with one
+ * term per remaining group folded on.  Floating-point addition is monotone in
+ * each argument, so folding on, group by group, the smallest d of each
+ * remaining group gives a value no leaf below can undercut, and folding on the
+ * largest c of each gives a value no leaf below can exceed.  A node is cut
+ *   (i)  when that smallest reachable d is above the budget, or
+ *   (ii) when that largest reachable c is strictly below the best c so far;
+ * nothing else is cut and no tolerance is involved, so the result is the
+ * enumeration's.  This is slow when the budget admits many assignments; the
+ * tests use it where it is not (tight budgets, moderate J) and
+ * orc_select_dp_integer for large J. */
 typedef struct {
     int J;
     const int *P;
     const long long *off;
     const double *c, *d;
     double budget;
-    double *base_d_suffix, *base_c_suffix; /* sums over groups >= j of the min-d option */
-    orc_seg *segs; int nsegs;              /* all hull increments, sorted by slope desc */
+    double *min_d, *max_c;   /* per group */
     int *p, *bp; int have; double bc, bd;
     long long nodes, node_limit;
 } orc_bnb;
-
-static int orc_seg_cmp(const void *a, const void *b) {
-    double sa = ((const orc_seg *)a)->slope, sb = ((const orc_seg *)b)->slope;
-    return (sa < sb) - (sa > sb);
-}
-
-static double orc_lp_bound(const orc_bnb *s, int j, double room) {
-    /* room = budget left after the min-d options of groups >= j */
-    double ub = 0.0;
-    for (int i = 0; i < s->nsegs && room > 0.0; ++i) {
-        const orc_seg *g = &s->segs[i];
-        if (g->j < j) continue;
-        if (g->dd <= room) { ub += g->dc; room -= g->dd; }
-        else { ub += g->dc * (room / g->dd); room = 0.0; }
-    }
-    return ub;
-}
 
 static void orc_bnb_rec(orc_bnb *s, int j, double cs, double ds) {
     if (s->nodes++ > s->node_limit) return;
@@ -431,17 +419,10 @@ static void orc_bnb_rec(orc_bnb *s, int j, double cs, double ds) {
         return;
     }
     {
-        double mind = ds + s->base_d_suffix[j];
-        double margin = 1e-9 * (fabs(mind) + fabs(s->budget)) + 1e-300;
-        if (mind > s->budget + margin) return;
-        if (s->have) {
-            double room = s->budget - mind;
-            if (room < 0.0) room = 0.0;
-            room += margin;
-            double ub = cs + s->base_c_suffix[j] + orc_lp_bound(s, j, room);
-            double m2 = 1e-9 * (fabs(ub) + fabs(s->bc)) + 1e-300;
-            if (ub + m2 < s->bc) return;
-        }
+        double lo_d = ds, hi_c = cs;
+        for (int k = j; k < s->J; ++k) { lo_d += s->min_d[k]; hi_c += s->max_c[k]; }
+        if (lo_d > s->budget) return;            /* (i)  */
+        if (s->have && hi_c < s->bc) return;     /* (ii) */
     }
     for (int p = 0; p < s->P[j]; ++p) {
         s->p[j] = p;
@@ -454,75 +435,19 @@ int orc_select_bnb(int J, const int *P, const long long *off, const double *c, c
                    double budget, long long node_limit, int *p_out, double *c_out,
                    double *d_out) {
     orc_bnb s;
-    int total = 0, rc;
+    int rc;
     memset(&s, 0, sizeof s);
     s.J = J; s.P = P; s.off = off; s.c = c; s.d = d; s.budget = budget;
     s.node_limit = node_limit > 0 ? node_limit : 2000000000LL;
-    for (int j = 0; j < J; ++j) total += P[j];
-    s.base_d_suffix = (double *)calloc((size_t)J + 1, sizeof(double));
-    s.base_c_suffix = (double *)calloc((size_t)J + 1, sizeof(double));
-    s.segs = (orc_seg *)calloc((size_t)total + 1, sizeof(orc_seg));
+    s.min_d = (double *)calloc((size_t)J + 1, sizeof(double));
+    s.max_c = (double *)calloc((size_t)J + 1, sizeof(double));
     s.p = (int *)calloc((size_t)J + 1, sizeof(int));
     s.bp = (int *)calloc((size_t)J + 1, sizeof(int));
-    int *greedy = (int *)calloc((size_t)J + 1, sizeof(int));
-    double *base_d = (double *)calloc((size_t)J + 1, sizeof(double));
-    double *base_c = (double *)calloc((size_t)J + 1, sizeof(double));
-    /* per group: min-d option (ties: larger c), then the upper convex hull */
     for (int j = 0; j < J; ++j) {
-        const double *cj = c + off[j], *dj = d + off[j];
-        int n = P[j], b = 0;
-        for (int p = 1; p < n; ++p)
-            if (dj[p] < dj[b] || (dj[p] == dj[b] && cj[p] > cj[b])) b = p;
-        base_d[j] = dj[b]; base_c[j] = cj[b]; greedy[j] = b;
-        /* gift-wrapping from the base point: repeatedly take the option with
-         * the steepest positive slope, ties to the farther point */
-        int cur = b;
-        for (;;) {
-            int nxt = -1; double best = 0.0;
-            for (int p = 0; p < n; ++p) {
-                double dd = dj[p] - dj[cur], dc = cj[p] - cj[cur];
-                if (dd <= 0.0 || dc <= 0.0) continue;
-                double sl = dc / dd;
-                if (nxt < 0 || sl > best || (sl == best && dj[p] > dj[nxt])) { nxt = p; best = sl; }
-            }
-            if (nxt < 0) break;
-            s.segs[s.nsegs].dd = dj[nxt] - dj[cur];
-            s.segs[s.nsegs].dc = cj[nxt] - cj[cur];
-            s.segs[s.nsegs].slope = best;
-            s.segs[s.nsegs].j = j;
-            s.segs[s.nsegs].to = nxt;
-            s.nsegs++;
-            cur = nxt;
-        }
-    }
-    for (int j = J - 1; j >= 0; --j) {
-        s.base_d_suffix[j] = s.base_d_suffix[j + 1] + base_d[j];
-        s.base_c_suffix[j] = s.base_c_suffix[j + 1] + base_c[j];
-    }
-    qsort(s.segs, (size_t)s.nsegs, sizeof(orc_seg), orc_seg_cmp);
-    /* incumbent: round the linear relaxation down (take hull increments by
-     * slope while they fit, a group stops at its first increment that does
-     * not), else the all-min-d assignment; both evaluated with the exact folds */
-    for (int pass = 0; pass < 2 && !s.have; ++pass) {
-        double cs = 0.0, ds = 0.0;
-        if (pass == 0) {
-            double room = budget - s.base_d_suffix[0];
-            int *blocked = (int *)calloc((size_t)J + 1, sizeof(int));
-            memcpy(s.p, greedy, sizeof(int) * (size_t)J);
-            for (int i = 0; i < s.nsegs; ++i) {
-                const orc_seg *g = &s.segs[i];
-                if (blocked[g->j]) continue;
-                if (g->dd <= room) { room -= g->dd; s.p[g->j] = g->to; }
-                else blocked[g->j] = 1;
-            }
-            free(blocked);
-        } else {
-            memcpy(s.p, greedy, sizeof(int) * (size_t)J);
-        }
-        for (int j = 0; j < J; ++j) { ds += d[off[j] + s.p[j]]; cs += c[off[j] + s.p[j]]; }
-        if (ds <= budget) {
-            s.have = 1; s.bc = cs; s.bd = ds;
-            memcpy(s.bp, s.p, sizeof(int) * (size_t)J);
+        s.min_d[j] = d[off[j]]; s.max_c[j] = c[off[j]];
+        for (int p = 1; p < P[j]; ++p) {
+            if (d[off[j] + p] < s.min_d[j]) s.min_d[j] = d[off[j] + p];
+            if (c[off[j] + p] > s.max_c[j]) s.max_c[j] = c[off[j] + p];
         }
     }
     orc_bnb_rec(&s, 0, 0.0, 0.0);
@@ -532,7 +457,57 @@ int orc_select_bnb(int J, const int *P, const long long *off, const double *c, c
         memcpy(p_out, s.bp, sizeof(int) * (size_t)J);
         *c_out = s.bc; *d_out = s.bd;
     }
-    free(s.base_d_suffix); free(s.base_c_suffix); free(s.segs); free(s.p); free(s.bp);
-    free(greedy); free(base_d); free(base_c);
+    free(s.min_d); free(s.max_c); free(s.p); free(s.bp);
     return rc;
+}
+
+/* The same integer program when every d is a non-negative integer: the
+ * textbook dynamic program of the multiple-choice knapsack over the integer
+ * budget.  best[w] after group j = the largest left-fold c over assignments of
+ * groups 0..j whose d sums to exactly w (integers: that sum has no rounding and
+ * no order).  best[w] + c_{j,p} is the left fold of the extended assignment,
+ * and because floating-point addition is monotone the largest prefix value
+ * gives the largest extended value, so the table holds true maxima of left
+ * folds.  Answer: the largest best[w] over w <= budget, the smallest such w,
+ * and one assignment that attains them (which one, among several with the same
+ * (c, d), is not specified).  Returns 0 ok, 1 infeasible, 3 too large. */
+int orc_select_dp_integer(int J, const int *P, const long long *off, const double *c,
+                          const long long *d, long long budget, int *p_out, double *c_out,
+                          long long *d_out) {
+    if (budget < 0) return 1;
+    if (budget > 50000000LL || (double)(budget + 1) * (double)(J + 1) > 4e8) return 3;
+    const size_t W = (size_t)budget + 1;
+    double *best = (double *)malloc(W * sizeof(double));
+    double *next = (double *)malloc(W * sizeof(double));
+    char *ok = (char *)calloc(W, 1), *nok = (char *)calloc(W, 1);
+    int *choice = (int *)malloc(W * (size_t)(J > 0 ? J : 1) * sizeof(int)); /* [j][w]: p that gave next[w] */
+    ok[0] = 1; best[0] = 0.0;
+    for (int j = 0; j < J; ++j) {
+        memset(nok, 0, W);
+        for (size_t w = 0; w < W; ++w) {
+            if (!ok[w]) continue;
+            for (int p = 0; p < P[j]; ++p) {
+                long long dv = d[off[j] + p];
+                if (dv < 0 || (long long)w + dv > budget) continue;
+                size_t w2 = w + (size_t)dv;
+                double v = best[w] + c[off[j] + p];
+                if (!nok[w2] || v > next[w2]) { nok[w2] = 1; next[w2] = v; choice[(size_t)j * W + w2] = p; }
+            }
+        }
+        { double *t = best; best = next; next = t; char *u = ok; ok = nok; nok = u; }
+    }
+    int have = 0; size_t bw = 0;
+    for (size_t w = 0; w < W; ++w)
+        if (ok[w] && (!have || best[w] > best[bw])) { have = 1; bw = w; }
+    if (have) {
+        *c_out = best[bw]; *d_out = (long long)bw;
+        size_t w = bw;
+        for (int j = J - 1; j >= 0; --j) {
+            int p = choice[(size_t)j * W + w];
+            p_out[j] = p;
+            w -= (size_t)d[off[j] + p];
+        }
+    }
+    free(best); free(next); free(ok); free(nok); free(choice);
+    return have ? 0 : 1;
 }

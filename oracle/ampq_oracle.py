@@ -79,6 +79,10 @@ def lib():
         L.orc_select_bnb.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_double, C.c_longlong, C.c_void_p, C.POINTER(C.c_double),
                                      C.POINTER(C.c_double)]
+        L.orc_select_dp_integer.restype = C.c_int
+        L.orc_select_dp_integer.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_longlong, C.c_void_p, C.POINTER(C.c_double),
+                                            C.POINTER(C.c_longlong)]
         _lib = L
     return _lib
 
@@ -251,8 +255,28 @@ def select_bruteforce(c_tables, d_tables, budget: float):
     return p[:J].copy(), co.value, do.value
 
 
+def select_dp_integer(c_tables, d_int_tables, budget: int):
+    """The integer program with integer-valued d by the textbook dynamic
+    program over the budget.  Returns (p[J], c, d) -- p is one optimal
+    assignment, not necessarily the lexicographically smallest -- or None."""
+    P, off, c, _ = _flatten(c_tables, d_int_tables)
+    d = np.ascontiguousarray(np.concatenate([np.asarray(x) for x in d_int_tables]) if len(P) else np.zeros(1),
+                             dtype=np.int64)
+    J = len(P)
+    p = np.zeros(max(J, 1), dtype=np.int32)
+    co, do = C.c_double(), C.c_longlong()
+    rc = lib().orc_select_dp_integer(J, _ptr(P), _ptr(off), _ptr(c), _ptr(d), int(budget), _ptr(p),
+                                     C.byref(co), C.byref(do))
+    if rc == 1:
+        return None
+    if rc:
+        raise RuntimeError("integer budget too large for the oracle's dynamic program")
+    return p[:J].copy(), co.value, int(do.value)
+
+
 def select_bnb(c_tables, d_tables, budget: float, node_limit: int = 0):
-    """Branch and bound with the same sums and ordering as the enumeration."""
+    """Plain depth-first branch and bound with the same sums and ordering as the
+    enumeration; slow when the budget admits many assignments."""
     P, off, c, d = _flatten(c_tables, d_tables)
     J = len(P)
     p = np.zeros(max(J, 1), dtype=np.int32)

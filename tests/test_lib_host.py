@@ -86,18 +86,44 @@ def test_select_absorbing_magnitudes(ampq, orc):
 
 
 @pytest.mark.parametrize("J,P", [(64, 2), (80, 2), (32, 16)])
-def test_select_large_matches_branch_and_bound(ampq, orc, J, P):
+def test_select_large_matches_integer_dynamic_program(ampq, orc, J, P):
+    """Sizes of the format/budget sweep (64 sub-graphs), of the 70B-shaped model
+    (80) and of many-column groups: loss MSEs on an integer grid, so that the
+    oracle's textbook dynamic program over the budget -- a method that shares
+    nothing with the library's solver -- gives the exact optimum.  (c, d) must
+    match; the library's assignment must attain them within the budget."""
     rng = np.random.default_rng(43)
+    c = [np.concatenate([[0.0], np.sort(rng.uniform(0.5, 2.0, P - 1))]) for _ in range(J)]
+    d = [np.concatenate([[0], np.sort((rng.uniform(0, 1, P - 1) ** 2 * 2000).astype(np.int64))]) for _ in range(J)]
+    df = [t.astype(float) for t in d]
+    hi = int(sum(t[-1] for t in d))
+    prev = -1.0
+    for frac in (0.01, 0.05, 0.2, 0.5):
+        budget = int(frac * hi)
+        ref = orc.select_dp_integer(c, d, budget)
+        got = ampq.select_tables(c, df, float(budget))
+        assert got[1] == ref[1] and got[2] == float(ref[2]), (frac, got[1:], ref[1:])
+        cs = ds = 0.0
+        for j, pj in enumerate(got[0]):
+            ds += df[j][pj]
+            cs += c[j][pj]
+        assert (cs, ds) == (got[1], got[2]) and ds <= budget and got[1] >= prev
+        prev = got[1]
+
+
+@pytest.mark.parametrize("J,P,fracs", [(40, 2, (0.012, 0.06, 0.15)), (24, 4, (0.01, 0.03)), (64, 2, (0.0015, 0.01, 0.03)), (80, 2, (0.01,))])
+def test_select_matches_plain_branch_and_bound(ampq, orc, J, P, fracs):
+    """Real-valued loss MSEs beyond the reach of the enumeration, at budgets tight
+    enough for the oracle's plain depth-first search: the assignment itself,
+    tie-break included, must match."""
+    rng = np.random.default_rng(45)
     c = [np.concatenate([[0.0], np.sort(rng.uniform(0.5, 2.0, P - 1))]) for _ in range(J)]
     d = [np.concatenate([[0.0], np.sort(rng.uniform(0, 1, P - 1) ** 2)]) for _ in range(J)]
     hi = sum(t[-1] for t in d)
-    prev = -1.0
-    for frac in (0.01, 0.05, 0.2, 0.5):
-        ref = orc.select_bnb(c, d, frac * hi, 50_000_000)
+    for frac in fracs:
+        ref = orc.select_bnb(c, d, frac * hi, 400_000_000)
         got = ampq.select_tables(c, d, frac * hi)
         assert got[0].tolist() == ref[0].tolist() and got[1] == ref[1] and got[2] == ref[2]
-        assert got[2] <= frac * hi and got[1] >= prev
-        prev = got[1]
 
 
 def test_select_edge_cases(ampq):

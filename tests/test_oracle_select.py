@@ -123,3 +123,69 @@ def test_branch_and_bound_large_and_absorbing(orc):
         ref = orc.select_bruteforce(c, d, frac * hi)
         got = orc.select_bnb(c, d, frac * hi)
         assert got[0].tolist() == ref[0].tolist() and got[1:] == ref[1:]
+
+
+def _fold(c_tabs, d_tabs, p):
+    c = d = 0.0
+    for j, pj in enumerate(p):
+        d += d_tabs[j][pj]
+        c += c_tabs[j][pj]
+    return c, d
+
+
+def test_integer_dynamic_program_matches_enumeration(orc):
+    """The integer-d dynamic program against the enumeration: same (c, d), and
+    its assignment is feasible and attains them (which of several equal
+    assignments it returns is not specified)."""
+    rng = np.random.default_rng(27)
+    for it in range(200):
+        J = int(rng.integers(1, 10))
+        c_tabs, d_tabs = [], []
+        for _ in range(J):
+            P = int(rng.integers(1, 5))
+            c = rng.uniform(0, 2, P) if it % 2 else rng.integers(0, 4, P).astype(float)
+            d = rng.integers(0, 30, P)
+            if rng.random() < 0.6:
+                c[0], d[0] = 0.0, 0
+            c_tabs.append(c)
+            d_tabs.append(d)
+        hi = int(sum(max(t) for t in d_tabs))
+        for budget in (0, hi // 20, hi // 3, (2 * hi) // 3, hi, 2 * hi + 1):
+            ref = orc.select_bruteforce(c_tabs, [t.astype(float) for t in d_tabs], float(budget))
+            got = orc.select_dp_integer(c_tabs, d_tabs, budget)
+            if ref is None:
+                assert got is None
+                continue
+            assert got[1] == ref[1] and got[2] == ref[2], (it, budget)
+            assert _fold(c_tabs, d_tabs, got[0]) == (ref[1], float(ref[2]))
+
+
+def test_integer_dynamic_program_absorbing_gains(orc):
+    """Gains spread over many orders of magnitude (small ones absorbed by
+    rounding): the dynamic program still holds the enumeration's left-fold maximum."""
+    rng = np.random.default_rng(28)
+    for _ in range(10):
+        J = 14
+        c = [np.array([0.0, float(x)]) for x in 10.0 ** rng.uniform(-17, 1, J)]
+        d = [np.array([0, int(x)]) for x in rng.integers(1, 50, J)]
+        hi = int(sum(t[1] for t in d))
+        for budget in (hi // 50, hi // 5, hi // 2):
+            ref = orc.select_bruteforce(c, [t.astype(float) for t in d], float(budget))
+            got = orc.select_dp_integer(c, d, budget)
+            assert got[1] == ref[1] and got[2] == ref[2]
+
+
+def test_branch_and_bound_moderate_sizes_against_dynamic_program(orc):
+    """Two independent exact methods beyond the reach of the enumeration: the
+    plain depth-first search and the integer dynamic program agree on (c, d) at
+    J = 40 binary groups with tight budgets."""
+    rng = np.random.default_rng(29)
+    J = 40
+    c = [np.array([0.0, float(x)]) for x in rng.uniform(0.5, 2.0, J)]
+    d = [np.array([0, int(x)]) for x in rng.integers(1, 1000, J)]
+    hi = int(sum(t[1] for t in d))
+    for budget in (hi // 100, hi // 30):
+        a = orc.select_bnb(c, [t.astype(float) for t in d], float(budget), 200_000_000)
+        b = orc.select_dp_integer(c, d, budget)
+        assert a[1] == b[1] and a[2] == b[2]
+        assert _fold(c, d, b[0]) == (a[1], a[2])
