@@ -304,6 +304,16 @@ int ampq_select_tables(int J, const int *P, const long long *off, const double *
                        const double *d, double budget, int *p_out, double *c_total,
                        double *d_total);
 
+/* Calibration split over several processes by SAMPLE: every entry of a
+ * per-layer table (s_l, d_model_{l,f}, d_meas_{l,f}) is a mean over calibration
+ * samples (Sec. 2.2: s_l = (1/R) sum_r s_l^r), so the value over all samples is
+ * the R-weighted mean of the per-process values.  tables is [nranks][L][K]
+ * row-major (process i's table computed over its R_local[i] samples), out is
+ * [L][K]: out = sum_i R_local[i] * tables[i] / sum_i R_local[i], the sum taken
+ * in order i = 0..nranks-1.  Host pointers; no context, no GPU. */
+int ampq_merge_sample_tables(const double *tables, const int *R_local, int nranks, int L, int K,
+                             double *out);
+
 /* Partition of a model's computation graph into sequential sub-graphs
  * (Appendix B, Algorithm 2).  Vertices 0..n-1, directed edges edge_src[e] ->
  * edge_dst[e]; the graph must be acyclic with exactly one sink (the end

@@ -22,6 +22,9 @@ shares nothing with the library.  Small inputs only (pure-Python loops).
                           given order while the loss-MSE budget holds, stopping
                           at the first that does not fit.  Prefix = the model's
                           own order; Random = a permutation the caller draws.
+  * merge_sample_tables(...)  per-layer means over all calibration samples from
+                          per-process means over disjoint sample sets (Sec. 2.2:
+                          s_l = (1/R) sum_r s_l^r): the R-weighted mean.
 """
 from __future__ import annotations
 
@@ -101,3 +104,18 @@ def select_in_order(order, d_low, c_low, budget):
         else:
             break
     return chosen, c, d
+
+
+def merge_sample_tables(tables, R_local):
+    """tables[i][l][k]: mean over process i's R_local[i] samples.  Returns the
+    mean over all samples, [l][k]."""
+    total = float(sum(R_local))
+    L, K = len(tables[0]), len(tables[0][0])
+    out = [[0.0] * K for _ in range(L)]
+    for l in range(L):
+        for k in range(K):
+            acc = 0.0
+            for i, R in enumerate(R_local):
+                acc += float(R) * tables[i][l][k]
+            out[l][k] = acc / total
+    return out

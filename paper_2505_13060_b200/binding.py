@@ -38,7 +38,7 @@ EXPORTS = [
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
     "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal", "ampq_set_measured",
-    "ampq_set_sharing", "ampq_get_pass_bytes",
+    "ampq_set_sharing", "ampq_get_pass_bytes", "ampq_merge_sample_tables",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -98,6 +98,7 @@ def lib():
     L.ampq_gain_table.argtypes = [i, i, vp, vp, vp, vp, vp, i, vp, i, vp]
     L.ampq_select_in_order.argtypes = [i, vp, vp, vp, C.c_double, vp, dp, dp]
     L.ampq_group_costs_table.argtypes = [vp, i, vp, i, vp, i, i, vp]
+    L.ampq_merge_sample_tables.argtypes = [vp, vp, i, i, i, vp]
     L.ampq_budget_from_tau.argtypes = [C.c_double, vp, i, dp]
     L.ampq_all_lowp_cost.argtypes = [vp, i, i, dp]
     L.ampq_select.argtypes = [vp, i, C.c_double, vp, dp, dp]
@@ -181,6 +182,20 @@ def group_costs_table(layer_ids, Q, d_layer) -> np.ndarray:
                                       d_layer.shape[1], _np_ptr(out))
     if rc:
         raise AmpqError(rc, "ampq_group_costs_table")
+    return out
+
+
+def merge_sample_tables(tables, R_local) -> np.ndarray:
+    """tables: [nranks, L, K] per-process tables of per-layer means over each
+    process's own samples; R_local: [nranks] sample counts.  Returns the [L, K]
+    table over all samples."""
+    t = np.ascontiguousarray(tables, dtype=np.float64)
+    R = np.ascontiguousarray(R_local, dtype=np.int32)
+    assert t.ndim == 3 and R.size == t.shape[0]
+    out = np.zeros(t.shape[1:])
+    rc = lib().ampq_merge_sample_tables(_np_ptr(t), _np_ptr(R), t.shape[0], t.shape[1], t.shape[2], _np_ptr(out))
+    if rc:
+        raise AmpqError(rc, "ampq_merge_sample_tables")
     return out
 
 

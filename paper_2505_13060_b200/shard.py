@@ -94,21 +94,23 @@ def reduce_amax(local_amax, group=None, device=None) -> np.ndarray:
     return a
 
 
-def merge_sample_rows(local_table, R_local: int, group=None, device=None) -> np.ndarray:
+def merge_sample_rows(binding, local_table, R_local: int, group=None, device=None) -> np.ndarray:
     """``local_table``: [L, 1 + 2F] rows (``layer_row``) computed over this rank's
-    ``R_local`` samples.  Every entry is a mean over samples, so the value over
-    all samples is the R-weighted mean over ranks: one SUM all-reduce of
-    [R_local * rows | R_local]."""
+    ``R_local`` samples.  The tables and sample counts of all ranks are gathered
+    (a few KB) and ``ampq_merge_sample_tables`` forms the table over all samples
+    on every rank, from the same inputs in the same order: bit-identical."""
     import torch
     import torch.distributed as dist
 
     tab = np.ascontiguousarray(local_table, dtype=np.float64)
     if not (dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1):
-        return tab
-    buf = np.concatenate([(tab * float(R_local)).reshape(-1), [float(R_local)]])
-    t = torch.from_numpy(buf)
+        return binding.merge_sample_tables(tab[None], [R_local])
+    world = dist.get_world_size(group)
+    mine = torch.from_numpy(np.concatenate([tab.reshape(-1), [float(R_local)]]))
     if device is not None:
-        t = t.to(device)
-    dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
-    out = t.cpu().numpy()
-    return out[:-1].reshape(tab.shape) / out[-1]
+        mine = mine.to(device)
+    parts = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(parts, mine, group=group)
+    parts = [p.cpu().numpy() for p in parts]
+    tables = np.stack([p[:-1].reshape(tab.shape) for p in parts])
+    return binding.merge_sample_tables(tables, [int(p[-1]) for p in parts])

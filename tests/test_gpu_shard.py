@@ -55,7 +55,7 @@ def test_two_sample_shards_equal_one_context(ampq, orc):
                 ctx.set_amax(lid, op, float(amax[k, op]))
         ctx.score()
         tables.append((np.stack([shard.layer_row(ctx.get_layer(i), F) for i in ids]), Rl))
-    merged = sum(t * R for t, R in tables) / sum(R for _, R in tables)   # what merge_sample_rows computes
+    merged = ampq.merge_sample_tables(np.stack([t for t, _ in tables]), [R for _, R in tables])   # what merge_sample_rows calls
     one = ampq.Context(0, st)
     oid = []
     for lt in lts:

@@ -103,6 +103,19 @@ def test_baselines_match_oracle_and_never_beat_the_integer_program(ampq):
                                            None, None) == ampq.ERR_INVALID   # not a permutation
 
 
+def test_merge_sample_tables_matches_oracle(ampq):
+    rng = np.random.default_rng(11)
+    for nranks, L, K in ((1, 4, 5), (2, 7, 5), (5, 3, 7)):
+        tables = rng.uniform(0, 3, (nranks, L, K)) * 10.0 ** rng.integers(-6, 3, (nranks, L, 1))
+        R = rng.integers(1, 9, nranks)
+        got = ampq.merge_sample_tables(tables, R)
+        assert got.tolist() == ho.merge_sample_tables(tables.tolist(), R.tolist())
+    with pytest.raises(ampq.AmpqError):
+        ampq.merge_sample_tables(np.zeros((2, 1, 1)), [0, 0])     # no samples at all
+    with pytest.raises(ampq.AmpqError):
+        ampq.merge_sample_tables(np.zeros((2, 1, 1)), [1, -1])
+
+
 def test_saved_layer_table_round_trips_bit_for_bit(ampq, tmp_path):
     from paper_2505_13060_b200 import shard, table
 

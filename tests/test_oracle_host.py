@@ -137,3 +137,27 @@ def test_baseline_strategies_hand_examples_and_bound():
         for order in (list(range(L)), rng.permutation(L).tolist()):
             ch, cs, ds = ho.select_in_order(order, d, c, budget)
             assert ds <= budget and cs <= best + 1e-12
+
+
+def test_merge_of_sample_means_equals_the_mean_over_all_samples():
+    """Pin (Sec. 2.2, s_l = (1/R) sum_r s_l^r): per-sample values with few
+    significant bits, so that every sum below is exact in double; the merge of
+    the per-shard means over unequal shards (3, 1 and 4 samples) must then equal
+    the mean over all 8 samples exactly, computed here with rationals."""
+    from fractions import Fraction
+
+    import random
+
+    rnd = random.Random(5)
+    L, K, shards = 3, 5, [3, 1, 4]
+    per_sample = [[[Fraction(rnd.randrange(0, 1 << 12), 1 << 6) * 24 for _ in range(K)] for _ in range(L)]
+                  for _ in range(sum(shards))]   # multiples of 24/64: divisible by 3, 4 and 8 without rounding
+    tables, r = [], 0
+    for n in shards:
+        tables.append([[float(sum(per_sample[r + i][l][k] for i in range(n)) / n) for k in range(K)] for l in range(L)])
+        r += n
+    want = [[float(sum(s[l][k] for s in per_sample) / len(per_sample)) for k in range(K)] for l in range(L)]
+    assert ho.merge_sample_tables(tables, shards) == want
+    # one shard is the identity; a shard without samples does not count
+    assert ho.merge_sample_tables([tables[0]], [3]) == tables[0]
+    assert ho.merge_sample_tables([tables[0], tables[1]], [3, 0]) == tables[0]

@@ -68,7 +68,7 @@ def worker(rank, world, port, out):
     amax = shard.reduce_amax(a)
     R_local = 3 if rank == 0 else 5
     rows = np.array([[1.0, 0.0, 2.0, 0.0, 4.0], [8.0, 0.0, 1.0, 0.0, 0.5]]) * (rank + 1)
-    merged = shard.merge_sample_rows(rows, R_local)
+    merged = shard.merge_sample_rows(binding, rows, R_local)
     dist.barrier()
     dist.destroy_process_group()
     with open(os.path.join(out, "rank%d.json" % rank), "w") as f:
