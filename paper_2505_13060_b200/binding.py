@@ -245,6 +245,7 @@ class Context:
             raise AmpqError(rc, "ampq_create")
         self.F = 2
         self._R = {}
+        self.device, self.stream = device, stream   # the cudaStream_t handle every call of this context runs on
 
     def _check(self, rc: int):
         if rc:

@@ -9,7 +9,12 @@ and a backward hook receives dL/dX and dL/dY; the sample's weight gradient
 dL/dW = dL/dY^T X is formed by a torch matmul (the GEMM that produces a gradient
 is not part of the scoring path) and both operands of the layer are streamed to
 ``ampq_stream_sample``, so the R per-sample weight gradients never exist at the
-same time.  Everything the method computes happens in the CUDA library; this
+same time: a sample's tensors are released as soon as the library's work on
+them is ordered before any reuse of their memory -- at once when the context
+runs on torch's current stream (the caching allocator hands a freed block only
+to later work of the same stream), else when a CUDA event recorded on the
+context's stream after the sample has completed, with at most two samples
+pending.  Everything the method computes happens in the CUDA library; this
 module only moves pointers.
 
 ``quantised(...)`` runs the model with chosen layers' inputs and weights replaced
@@ -46,8 +51,28 @@ class Calibrator:
                 self.layer_ids.append(ctx.register_layer(ampq.BGEMM, name, R))
         self._r = None
         self._x = {}
-        self._keep = []   # tensors borrowed by the library until the stream has caught up
+        self._keep = []      # tensors the library borrowed during the current sample
+        self._pending = []   # (event on the context's stream, tensors) of earlier samples
         self._handles = []
+
+    # -- lifetime of borrowed tensors -------------------------------------------
+    def _same_stream(self) -> bool:
+        return torch.cuda.current_stream().cuda_stream == self.ctx.stream
+
+    def _release_sample(self):
+        """Called when a sample's block ends: nothing more will be launched on its tensors."""
+        if not self._keep:
+            return
+        if self._same_stream():
+            self._keep = []   # stream order protects the memory
+            return
+        ev = torch.cuda.Event()
+        ev.record(torch.cuda.ExternalStream(self.ctx.stream))
+        self._pending.append((ev, self._keep))
+        self._keep = []
+        self._pending = [(e, t) for e, t in self._pending if not e.query()]
+        while len(self._pending) > 2:
+            self._pending.pop(0)[0].synchronize()
 
     # -- hooks ----------------------------------------------------------------
     def _fwd(self, idx):
@@ -60,6 +85,8 @@ class Calibrator:
         def hook(module, grad_input, grad_output):
             if self._r is None:
                 return
+            if not self._same_stream():   # the library's stream reads what torch's stream has just produced
+                torch.cuda.ExternalStream(self.ctx.stream).wait_stream(torch.cuda.current_stream())
             if isinstance(module, BatchedMatmul):   # both operands belong to the sample
                 lid = self.layer_ids[idx]
                 for k, (x, gx) in enumerate(zip(self._x.pop(idx), grad_input)):
@@ -99,11 +126,13 @@ class Calibrator:
         finally:
             self._r = None
             self._x.clear()
+            self._release_sample()
 
     def end(self):
         self.ctx.stream_end()
         res = [self.ctx.get_layer(lid) for lid in self.layer_ids]   # synchronises: the borrowed tensors are free
-        self._keep.clear()
+        self._keep = []
+        self._pending = []
         for h in self._handles:
             h.remove()
         self._handles = []
@@ -155,4 +184,6 @@ class Calibrator:
                 h.remove()
             for m, w in saved:
                 m.weight.data.copy_(w)
-            self._keep.clear()
+            if not self._same_stream():
+                torch.cuda.ExternalStream(self.ctx.stream).synchronize()
+            self._keep = []

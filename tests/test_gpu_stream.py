@@ -360,3 +360,43 @@ def test_attention_block_with_batched_products_through_hooks(ampq, orc):
     print("attention block: measured / predicted loss MSE = %.3f" % (measured / d_meas))
     assert 0.4 < measured / d_meas < 2.5, (measured, d_meas)
     ctx.destroy()
+
+
+@pytest.mark.parametrize("own_stream", [False, True])
+def test_hook_calibration_memory_does_not_grow_with_samples(ampq, orc, own_stream):
+    """Streaming calibration exists so that the R per-sample weight gradients
+    never live together: the peak device memory of a hooked calibration with
+    R = 24 samples stays at that of R = 3 (a kept gradient per sample would add
+    21 x 3 x 4 MiB here), whether the context runs on torch's stream or on one
+    of its own, and both give the same per-sample values."""
+    from paper_2505_13060_b200 import hooks
+
+    torch.manual_seed(1)
+    width, tokens = 1024, 32
+    model = torch.nn.Sequential(torch.nn.Linear(width, width), torch.nn.GELU(), torch.nn.Linear(width, width),
+                                torch.nn.GELU(), torch.nn.Linear(width, width)).cuda()
+    side = torch.cuda.Stream() if own_stream else None
+
+    def run(R):
+        xs = torch.randn(R, tokens, width, device="cuda")
+        ctx = ampq.Context(0, (side or torch.cuda.current_stream()).cuda_stream)
+        ctx.set_formats([0, E4M3])
+        cal = hooks.Calibrator(ctx, model, R)
+        torch.cuda.synchronize()
+        torch.cuda.reset_peak_memory_stats()
+        base = torch.cuda.memory_allocated()
+        cal.begin()
+        for r in range(R):
+            with cal.sample(r):
+                model(xs[r]).square().mean().backward()
+            model.zero_grad(set_to_none=True)
+        res = cal.end()
+        peak = torch.cuda.max_memory_allocated() - base
+        ctx.destroy()
+        return peak, res
+
+    run(2)   # warm the allocator and the library's workspace
+    small, res3 = run(3)
+    large, res24 = run(24)
+    assert large < small + 6 * width * width * 4, (small, large)
+    assert np.all(res24[1]["s_per_sample"] > 0)

@@ -14,6 +14,7 @@ import pytest
 import torch
 
 from helpers import REL_TOL, assert_close
+from paper_2505_13060_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
@@ -46,7 +47,7 @@ def _noalloc(ampq, values, grads, fmt, amax, out):
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_noalloc_matches_score_twice_in_a_row(ampq, dtype):
+def test_noalloc_matches_score_twice_in_a_row(ampq, orc, dtype):
     g = torch.Generator(device="cuda").manual_seed(11)
     out = torch.empty(3, dtype=torch.float64, device="cuda")
     cases = [(2 * 524288 + 12345, E4M3, -1.0), (70001, E5M2, -1.0), (524288, E4M3, 2.5), (7, E5M2, -1.0), (0, E4M3, -1.0)]
@@ -64,6 +65,11 @@ def test_noalloc_matches_score_twice_in_a_row(ampq, dtype):
             assert got[2] == want[2], (n, fmt, got, want)          # amax: exact
             assert_close(got[:2], want[:2], "no-alloc [S, D] n=%d fmt=%d" % (n, fmt), tol=REL_TOL)
         assert got1.tobytes() == got2.tobytes()
+        if n:   # and the oracle itself, not only the entry point that was checked against it
+            a, _, _, seg = orc.score_operand(synth.to_numpy(v).reshape(1, -1), synth.to_numpy(gr).reshape(1, -1), 1, True,
+                                             [fmt], amax_preset=None if amax < 0 else amax)
+            assert got1[2] == float(a)
+            assert_close(got1[:2], seg[0], "no-alloc against the oracle n=%d fmt=%d" % (n, fmt), tol=REL_TOL)
 
 
 def test_noalloc_refuses_what_does_not_fit(ampq):
