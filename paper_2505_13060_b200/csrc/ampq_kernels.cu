@@ -448,15 +448,29 @@ __device__ __forceinline__ void consumer_barrier() {  // the kConsumers scoring 
     asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
 }
 
-// Waits for a phase of an mbarrier, at most kSpinLimit polls.  A wait that runs
-// out raises the CTA's abort flag; once that is up every wait returns false
-// after one poll, so that all threads still walk the same control flow to the
-// end.
+// Polls and suspend hint of the stage waits (scoring warps waiting for a full
+// stage, the producer waiting for an empty one).  A test build
+// (-DAMPQ_TEST_SHORT_WAITS) makes them give up after a handful of polls, long
+// before the copy they wait for can land, to exercise the time-out path: every
+// copy still completes, because the producer's final drain below keeps the full
+// limit.
+#ifdef AMPQ_TEST_SHORT_WAITS
+constexpr unsigned kStageSpinLimit = 2u;
+constexpr unsigned kStageHintNs = 0u;
+#else
+constexpr unsigned kStageSpinLimit = kSpinLimit;
+constexpr unsigned kStageHintNs = 2000u;
+#endif
+
+// Waits for a phase of an mbarrier, at most kStageSpinLimit polls.  A wait that
+// runs out raises the CTA's abort flag; once that is up every wait returns
+// false after one poll, so that all threads still walk the same control flow to
+// the end.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* b, unsigned parity, volatile int* s_abort) {
-    if (mbar_try_wait(b, parity)) return true;
-    for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+    if (mbar_try_wait(b, parity, kStageHintNs)) return true;
+    for (unsigned spin = 0; spin < kStageSpinLimit; ++spin) {
         if (*s_abort) return false;
-        if (mbar_try_wait(b, parity)) return true;
+        if (mbar_try_wait(b, parity, kStageHintNs)) return true;
     }
     *s_abort = 1;
     return false;
@@ -742,93 +756,17 @@ __device__ __forceinline__ bool tile_in_bounds(const Tensor& tn, const TileGeom&
 #endif
 }
 
-// The scoring kernel.  Persistent: CTA b takes tiles b, b + gridDim.x, ... of
-// the launch's tile table.  Warps 0..7 score; warp 8 is the producer: one lane
-// streams every full 16-byte-aligned chunk of the value tile and of its RB
-// gradient tiles into a ring of shared-memory stages with bulk asynchronous
-// copies, running as far ahead as the ring is deep, tile after tile, so that
-// the bytes in flight do not depend on how long the arithmetic of a chunk
-// takes.  A scoring thread takes its 16-byte vectors of a stage into
-// registers, hands the stage back and then does the arithmetic.  fp32 sums are
-// flushed into fp64 every kFlushTerms terms; a tile ends with the CTA-wide
-// ordered sum and one partial per (sample, accumulator).
-//
-// One launch per element type DT and sample-group size RB (1..4): per-sample
-// operands and the single-sample remainder of shared operands run with RB = 1;
-// shared operands (weights) are read once per group of up to four samples.
+// The scoring warps' walk over the tiles of the launch (see score_kernel).
 template <int DT, int FMASK, int RB, bool CAUSAL>
-__global__ void __launch_bounds__(kScoreThreads, kScoreCtasPerSm)
-score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
-             int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
-             LaunchStatus* __restrict__ status, int out_stride) {
+__device__ __forceinline__ void score_tiles(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin,
+                                            long long ntiles, int tile_shift, const float* __restrict__ scales,
+                                            double* __restrict__ partials, LaunchStatus* __restrict__ status,
+                                            int out_stride, const unsigned char* ring, unsigned long long* full,
+                                            unsigned long long* empty, double* s_red, volatile int* s_abort) {
     using RG = Ring<RB>;
     constexpr int NACC = Fm<FMASK>::kAcc;
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* ring = smem;
-    unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + RG::kRingBytes);
-    unsigned long long* empty = full + RG::kStages;
-    double* s_red = reinterpret_cast<double*>(empty + RG::kStages);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(s_red + RG::kRedDoubles);
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < RG::kStages; ++s) {
-            mbar_init(full + s, 1);
-            mbar_init(empty + s, kConsumers / 32);
-        }
-        *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const bool producer = threadIdx.x >= kConsumers;
-    unsigned it = 0;  // chunks the producer has put into the ring so far
-    RingPos<RG::kStages> pos;  // both sides walk the ring in the same order
-    int t = 0;        // tensor of the current tile; tiles only move forward
-    if (producer) {
-        if (!CAUSAL && threadIdx.x == kConsumers) {  // causal tiles do not go through the ring
-            for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-                while (tile >= __ldg(tile_begin + t + 1)) ++t;
-                const Tensor& tn = tens[t];
-                const TileGeom q = tile_geometry<RB, CAUSAL>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
-                constexpr int es = Elem<DT>::kBytes;
-                const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
-                const char* gb[RB];
-                grad_bases<RB, es>(tn, q, gb);
-                bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
-#pragma unroll
-                for (int r = 0; r < RB; ++r) aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
-                const int nchunks = aligned && tile_in_bounds<RB>(tn, q) ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
-                for (int c = 0; c < nchunks; ++c) {
-                    // the stage must have been handed back once per earlier lap
-                    if (it >= (unsigned)RG::kStages && !mbar_wait(empty + pos.stage, pos.parity ^ 1u, s_abort)) break;
-                    unsigned char* dst = ring + pos.stage * RG::kStageBytes;
-                    mbar_arrive_expect_tx(full + pos.stage, RG::kStageBytes);
-                    bulk_load(dst, vb + (long long)c * RG::kChunkBytes, RG::kChunkBytes, full + pos.stage);
-#pragma unroll
-                    for (int r = 0; r < RB; ++r)
-                        bulk_load(dst + (1 + r) * RG::kChunkBytes, gb[r] + (long long)c * RG::kChunkBytes,
-                                  RG::kChunkBytes, full + pos.stage);
-                    pos.advance();
-                    ++it;
-                }
-                if (*s_abort) break;
-            }
-            if (*s_abort) {
-                // The scoring warps stopped taking stages.  Every copy issued so far
-                // must have landed before the CTA gives its shared memory back:
-                // wait (bounded) for the last lap of each stage.
-                for (unsigned k = 0; k < (unsigned)RG::kStages && k < it; ++k) {
-                    const unsigned j = it - 1 - k;
-                    for (unsigned spin = 0; spin < kSpinLimit; ++spin)
-                        if (mbar_try_wait(full + j % RG::kStages, (j / RG::kStages) & 1)) break;
-                }
-                atomicExch(&status->timeout, 1);
-            }
-        }
-        return;
-    }
-
-    // ---- scoring warps
+    RingPos<RG::kStages> pos;  // the same walk of the ring as the producer's
+    int t = 0;                 // tensor of the current tile; tiles only move forward
     int red_block = 0;
     for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         while (tile >= __ldg(tile_begin + t + 1)) ++t;
@@ -880,6 +818,100 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         reduce_and_store<NACC, RB>(acc64, s_red + red_block * (kConsumers / 32) * RB * NACC, partials, q.slot0,
                                    tn.stream_slot_stride, out_stride);
         red_block ^= 1;
+    }
+}
+
+// The scoring kernel.  Persistent: CTA b takes tiles b, b + gridDim.x, ... of
+// the launch's tile table.  Warps 0..7 score; warp 8 is the producer: one lane
+// streams every full 16-byte-aligned chunk of the value tile and of its RB
+// gradient tiles into a ring of shared-memory stages with bulk asynchronous
+// copies, running as far ahead as the ring is deep, tile after tile, so that
+// the bytes in flight do not depend on how long the arithmetic of a chunk
+// takes.  A scoring thread takes its 16-byte vectors of a stage into
+// registers, hands the stage back and then does the arithmetic.  fp32 sums are
+// flushed into fp64 every kFlushTerms terms; a tile ends with the CTA-wide
+// ordered sum and one partial per (sample, accumulator).
+//
+// One launch per element type DT and number RB (1..4) of gradient streams per
+// read of the values: per-sample operands and the single-sample remainder of
+// shared operands run with RB = 1; shared operands (weights) are read once per
+// group of up to four samples; a per-sample operand that several layers read is
+// read once per group of up to four layers.
+template <int DT, int FMASK, int RB, bool CAUSAL>
+__global__ void __launch_bounds__(kScoreThreads, kScoreCtasPerSm)
+score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, long long ntiles,
+             int tile_shift, const float* __restrict__ scales, double* __restrict__ partials,
+             LaunchStatus* __restrict__ status, int out_stride) {
+    using RG = Ring<RB>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* ring = smem;
+    unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + RG::kRingBytes);
+    unsigned long long* empty = full + RG::kStages;
+    double* s_red = reinterpret_cast<double*>(empty + RG::kStages);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_red + RG::kRedDoubles);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < RG::kStages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, kConsumers / 32);
+        }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const bool producer = threadIdx.x >= kConsumers;
+    unsigned it = 0;  // chunks the producer has put into the ring so far
+    RingPos<RG::kStages> pos;  // both sides walk the ring in the same order
+    int t = 0;        // tensor of the current tile; tiles only move forward
+    if (producer) {
+        if (!CAUSAL && threadIdx.x == kConsumers) {  // causal tiles do not go through the ring
+            for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+                while (tile >= __ldg(tile_begin + t + 1)) ++t;
+                const Tensor& tn = tens[t];
+                const TileGeom q = tile_geometry<RB, CAUSAL>(tn, (int)(tile - __ldg(tile_begin + t)), tile_shift);
+                constexpr int es = Elem<DT>::kBytes;
+                const char* vb = reinterpret_cast<const char*>(tn.values) + q.voff * es;
+                const char* gb[RB];
+                grad_bases<RB, es>(tn, q, gb);
+                bool aligned = (reinterpret_cast<uintptr_t>(vb) & 15) == 0;
+#pragma unroll
+                for (int r = 0; r < RB; ++r) aligned = aligned && (reinterpret_cast<uintptr_t>(gb[r]) & 15) == 0;
+                const int nchunks = aligned && tile_in_bounds<RB>(tn, q) ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
+                for (int c = 0; c < nchunks; ++c) {
+                    // the stage must have been handed back once per earlier lap
+                    if (it >= (unsigned)RG::kStages && !mbar_wait(empty + pos.stage, pos.parity ^ 1u, s_abort)) break;
+                    unsigned char* dst = ring + pos.stage * RG::kStageBytes;
+                    mbar_arrive_expect_tx(full + pos.stage, RG::kStageBytes);
+                    bulk_load(dst, vb + (long long)c * RG::kChunkBytes, RG::kChunkBytes, full + pos.stage);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+                        bulk_load(dst + (1 + r) * RG::kChunkBytes, gb[r] + (long long)c * RG::kChunkBytes,
+                                  RG::kChunkBytes, full + pos.stage);
+                    pos.advance();
+                    ++it;
+                }
+                if (*s_abort) break;
+            }
+        }
+    } else {
+        score_tiles<DT, FMASK, RB, CAUSAL>(tens, tile_begin, ntiles, tile_shift, scales, partials, status, out_stride,
+                                           ring, full, empty, s_red, s_abort);
+    }
+    // Every thread of the CTA meets here: the producer has stopped issuing and the
+    // scoring warps have stopped taking stages.  If a wait ran out on either side,
+    // every copy issued so far must still land before the CTA gives its shared
+    // memory back: the producer lane waits (bounded, at the full limit) for the
+    // last lap of each stage; a stage's earlier laps had completed before it was
+    // refilled.  Then the time-out is reported.
+    __syncthreads();
+    if (*s_abort && threadIdx.x == kConsumers) {
+        for (unsigned k = 0; k < (unsigned)RG::kStages && k < it; ++k) {
+            const unsigned j = it - 1 - k;
+            for (unsigned spin = 0; spin < kSpinLimit; ++spin)
+                if (mbar_try_wait(full + j % RG::kStages, (j / RG::kStages) & 1)) break;
+        }
+        atomicExch(&status->timeout, 1);
     }
 }
 
