@@ -98,12 +98,15 @@ struct SegmentJob {
     unsigned amax_bits;
     int flag;                      // 1: the tensor held Inf/NaN
     float scales[2 * kMaxLow];
+    unsigned amax_done;            // amax CTAs that have finished (the last one forms the scales)
 };
 
 struct LaunchStatus {
     int nonfinite;  // set when some tensor's amax is Inf/NaN
     int timeout;    // set when a wait inside the scoring kernel ran out
     int bounds;     // set by a -DAMPQ_BOUNDS_CHECK build when a tile falls outside its tensor
+    unsigned amax_done;      // amax CTAs that have finished: the last one forms the scales
+    unsigned finalize_done;  // finalize CTAs that have finished: the last one combines the layers
 };
 
 }  // namespace ampq

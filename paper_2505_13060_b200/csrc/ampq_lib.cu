@@ -4,6 +4,7 @@
 // path is in ampq_kernels.cu.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstdio>
@@ -158,6 +159,8 @@ struct ampq_ctx {
     DevBuf<SegmentJob> d_jobs;          // one job per (tensor, sample) of a streaming pass
     DevBuf<double> d_job_partials;      // per-tile partials of the job in flight (jobs are ordered on the stream)
     DevBuf<SegmentJob> d_fq_job;        // tables of a fake-quantisation call
+    std::vector<void*> retired;         // outgrown job-partial buffers, freed when no job can be in flight
+    size_t job_partials_hint = 0;       // doubles of the last job-partial allocation
 
     bool timing = false;            // record CUDA events around the kernels of a score
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
@@ -520,11 +523,17 @@ int stage_host_operands(ampq_ctx* ctx) {
     return AMPQ_OK;
 }
 
+void free_retired(ampq_ctx* ctx) {
+    for (void* p : ctx->retired) cudaFree(p);
+    ctx->retired.clear();
+}
+
 int sync_results(ampq_ctx* ctx) {
     if (!ctx->scored) return fail(ctx, AMPQ_ERR_STATE, "no score has been issued");
     if (ctx->pending) {
         AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
         ctx->pending = false;
+        free_retired(ctx);  // every job that could use them has finished
     }
     if (!ctx->tens.empty() && ctx->h_status.p->bounds)
         return fail(ctx, AMPQ_ERR_CUDA, "bounds check: a scoring tile fell outside its tensor (library bug); the results of this score are invalid");
@@ -589,21 +598,36 @@ int prepare_tables(ampq_ctx* ctx) {
     return AMPQ_OK;
 }
 
-// Per-layer combine and the asynchronous read-back of every small result.
-int combine_and_read_back(ampq_ctx* ctx, int T, int L, int S) {
-    const int nacc = ctx->F;
-    cudaStream_t st = ctx->stream;
+// alpha_f = 2^(-2 m_f)/12 (Sec. 2.2) and the accumulator column of every format.
+CombineParams combine_params(const ampq_ctx* ctx) {
     CombineParams prm{};
-    prm.nacc = nacc;
+    prm.nacc = ctx->F;
     for (int f = 1; f < ctx->F; ++f) {
         prm.alpha[f] = std::ldexp(1.0, -2 * mantissa_bits_of(ctx->fmt[f])) / 12.0;
         prm.acc_of_fmt[f] = 1 + ctx->slot_of_fmt[f];
     }
-    AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, prm, ctx->d_seg_out.p, ctx->d_layer_out.p, st), "combine");
-    ++ctx->launches;
-    (void)T;
-    (void)S;
-    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_arena.p, ctx->d_arena.p, ctx->arena_bytes, cudaMemcpyDeviceToHost, st), "D2H results");
+    return prm;
+}
+
+// The asynchronous read-back of every small result of a pass.
+int read_back(ampq_ctx* ctx) {
+    AMPQ_CUDA(cudaMemcpyAsync(ctx->h_arena.p, ctx->d_arena.p, ctx->arena_bytes, cudaMemcpyDeviceToHost, ctx->stream), "D2H results");
+    return AMPQ_OK;
+}
+
+// Per-tile partials of a streamed sample.  Jobs are ordered on the stream, so
+// one buffer serves them all; when a larger sample arrives the buffer grows
+// geometrically and the old one, which earlier jobs in flight may still use, is
+// kept until the pass ends instead of being freed (a free would synchronise).
+int ensure_job_partials(ampq_ctx* ctx, size_t n) {
+    if (n <= ctx->d_job_partials.cap) return AMPQ_OK;
+    if (ctx->d_job_partials.p) ctx->retired.push_back(ctx->d_job_partials.p);
+    ctx->d_job_partials.p = nullptr;
+    ctx->d_job_partials.cap = 0;
+    size_t want = n > 2 * ctx->job_partials_hint ? n : 2 * ctx->job_partials_hint;
+    AMPQ_CUDA(cudaMalloc(reinterpret_cast<void**>(&ctx->d_job_partials.p), want * sizeof(double)), "cudaMalloc(job partials)");
+    ctx->d_job_partials.cap = want;
+    ctx->job_partials_hint = want;
     return AMPQ_OK;
 }
 
@@ -613,9 +637,15 @@ int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, LaunchStatus* status, in
                         const void* grads, long long numel, float preset, long long ntiles) {
     cudaStream_t st = ctx->stream;
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
-    AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, st), "job_prepare");
-    AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st), "amax");
-    AMPQ_CUDA(launch_scales(1, ctx->fmask, &job->tensor, &job->amax_bits, job->scales, &job->flag, status, st, ctx->scale_pow2), "scales");
+    // with a preset the scales are formed while the tables are filled; otherwise by the last CTA of the amax pass
+    AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, ctx->fmask, ctx->scale_pow2, status, st), "job_prepare");
+    ++ctx->launches;
+    if (namax > 0) {
+        AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st,
+                              scales_args(1, ctx->fmask, &job->tensor, &job->amax_bits, job->scales, &job->flag, status,
+                                          ctx->scale_pow2, &job->amax_done)), "amax");
+        ++ctx->launches;
+    }
     return AMPQ_OK;
 }
 
@@ -668,7 +698,8 @@ int ampq_destroy(ampq_ctx* ctx) {
     if (!ctx) return AMPQ_OK;
     {
         DeviceGuard g(ctx->device);
-        if (ctx->pending) cudaStreamSynchronize(ctx->stream);
+        if (ctx->pending || !ctx->retired.empty()) cudaStreamSynchronize(ctx->stream);
+        free_retired(ctx);
         for (auto& l : ctx->layers)
             for (int k = 0; k < 2; ++k)
                 if (l.op[k].stage) cudaFree(l.op[k].stage);
@@ -847,15 +878,22 @@ int ampq_score(ampq_ctx* ctx) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
         ++ctx->launches;
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[1], st), "cudaEventRecord");
-        if (ctx->namax_tiles > 0 && ctx->measured) {
-            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
+        // scale and inverse scale of every tensor: by the last CTA of the amax pass, or, when
+        // nothing is measured, by a small launch of their own
+        const ScalesArgs sa = scales_args(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p,
+                                          ctx->d_status.p, ctx->scale_pow2, &ctx->d_status.p->amax_done);
+        const bool amax_pass = ctx->namax_tiles > 0 && ctx->measured;
+        if (amax_pass) {
+            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st, sa), "amax");
             ++ctx->launches;
         }
         if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched
             AMPQ_CUDA(cudaMemsetAsync(ctx->d_partials.p, 0, (size_t)ctx->nslots * nacc * sizeof(double), st), "memset partials");
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
-        AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
-        ++ctx->launches;
+        if (!amax_pass) {
+            AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
+            ++ctx->launches;
+        }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[3], st), "cudaEventRecord");
         for (int c = 0; c < kScoreClasses; ++c) {
             if (ctx->ntiles[c] <= 0) continue;
@@ -867,9 +905,14 @@ int ampq_score(ampq_ctx* ctx) {
             ++ctx->launches;
         }
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[4], st), "cudaEventRecord");
-        AMPQ_CUDA(launch_finalize(ctx->d_segs.p, S, nacc, ctx->d_partials.p, ctx->d_seg_out.p, st), "finalize");
-        ++ctx->launches;
-        if ((rc = combine_and_read_back(ctx, T, L, S))) return rc;
+        {   // ordered sums per segment; the CTA that finishes last combines the layers
+            CombineArgs ca;
+            ca.counter = &ctx->d_status.p->finalize_done;
+            ca.layers = ctx->d_lay.p; ca.L = L; ca.F = ctx->F; ca.prm = combine_params(ctx); ca.layer_out = ctx->d_layer_out.p;
+            AMPQ_CUDA(launch_finalize(ctx->d_segs.p, S, nacc, ctx->d_partials.p, ctx->d_seg_out.p, st, ca), "finalize");
+            ++ctx->launches;
+        }
+        if ((rc = read_back(ctx))) return rc;
         if (tm) {
             AMPQ_CUDA(cudaEventRecord(ctx->ev[5], st), "cudaEventRecord");
             ctx->ev_valid = true;
@@ -888,6 +931,10 @@ int ampq_stream_begin(ampq_ctx* ctx) {
     if (ctx->pending) {
         AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
         ctx->pending = false;
+    }
+    if (!ctx->retired.empty()) {  // left by a streaming pass that was never ended
+        AMPQ_CUDA(cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+        free_retired(ctx);
     }
     // tables over EVERY registered layer: tensor 2*l + operand, one segment per sample
     ctx->tens.clear(); ctx->segs.clear(); ctx->lay.clear(); ctx->scored_layer_ids.clear();
@@ -921,8 +968,19 @@ int ampq_stream_begin(ampq_ctx* ctx) {
     AMPQ_CUDA(ctx->d_lay.ensure(L), "cudaMalloc(layers)");
     AMPQ_CUDA(ctx->d_jobs.ensure(S), "cudaMalloc(jobs)");
     {
-        const int rc = ensure_results(ctx, T, S, nacc, (size_t)out_off);
+        int rc = ensure_results(ctx, T, S, nacc, (size_t)out_off);
         if (rc) return rc;
+        // room for the per-tile partials of the largest operand that is bound (a hint: samples
+        // of operands that are not bound, or larger ones, make the buffer grow later)
+        long long most = 0;
+        for (const auto& l : ctx->layers)
+            for (int k = 0; k < 2; ++k)
+                if (l.op[k].bound) {
+                    const long long ext = extent_of(l, l.op[k]);
+                    const int shift = pick_tile_shift(ext, ctx->max_ctas);
+                    most = std::max(most, (ext + (1LL << shift) - 1) >> shift);
+                }
+        if (most > 0 && most <= 0x7FFFFFFFLL && (rc = ensure_job_partials(ctx, (size_t)most * nacc + 1))) return rc;
     }
     cudaStream_t st = ctx->stream;
     if (L) AMPQ_CUDA(cudaMemcpyAsync(ctx->d_lay.p, ctx->lay.data(), L * sizeof(Layer), cudaMemcpyHostToDevice, st), "H2D layers");
@@ -959,7 +1017,7 @@ int ampq_stream_sample(ampq_ctx* ctx, int layer_id, int operand, int r, int dtyp
     const int shift = pick_tile_shift(numel, ctx->max_ctas);
     const long long ntiles = (numel + (1LL << shift) - 1) >> shift;
     if (ntiles > 0x7FFFFFFFLL) return fail(ctx, AMPQ_ERR_TOO_LARGE, "more than 2^31-1 tiles in one sample");
-    AMPQ_CUDA(ctx->d_job_partials.ensure((size_t)ntiles * nacc + 1), "cudaMalloc(job partials)");
+    if ((rc = ensure_job_partials(ctx, (size_t)ntiles * nacc + 1))) return rc;
     SegmentJob* job = ctx->d_jobs.p + seg;
     cudaStream_t st = ctx->stream;
     // S only: a preset of 0 keeps the amax pass away; the D columns of the slots are cleared instead of written
@@ -969,9 +1027,10 @@ int ampq_stream_sample(ampq_ctx* ctx, int layer_id, int operand, int r, int dtyp
         AMPQ_CUDA(cudaMemsetAsync(ctx->d_job_partials.p, 0, (size_t)ntiles * nacc * sizeof(double), st), "memset partials");
     AMPQ_CUDA(launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &job->tensor, job->tile_begin, 1, ntiles, shift, ctx->max_ctas,
                            ctx->measured ? ctx->fmask : 0, job->scales, ctx->d_job_partials.p, ctx->d_status.p, st, 0, nacc), "score");
-    AMPQ_CUDA(launch_finalize(&job->segment, 1, nacc, ctx->d_job_partials.p, ctx->d_seg_out.p + (size_t)seg * nacc, st), "finalize");
-    AMPQ_CUDA(launch_job_fold(job, tensor, ctx->d_amax_bits.p, ctx->d_flags.p, ctx->d_scales.p, st), "job_fold");
-    ctx->launches += numel > 0 ? 6 : 4;
+    if (ntiles > 0) ++ctx->launches;
+    AMPQ_CUDA(launch_job_finish(job, nacc, ctx->d_job_partials.p, ctx->d_seg_out.p + (size_t)seg * nacc, tensor,
+                                ctx->d_amax_bits.p, ctx->d_flags.p, ctx->d_scales.p, st), "job_finish");
+    ++ctx->launches;
     return AMPQ_OK;
 }
 
@@ -984,7 +1043,12 @@ int ampq_stream_end(ampq_ctx* ctx) {
     for (const auto& ly : ctx->lay) nseg += 2 * ly.R;
     const int T = (int)ctx->tens.size(), L = (int)ctx->lay.size();
     int rc = AMPQ_OK;
-    if (T > 0 && (rc = combine_and_read_back(ctx, T, L, nseg))) return rc;
+    if (T > 0) {
+        AMPQ_CUDA(launch_combine(ctx->d_lay.p, L, ctx->F, combine_params(ctx), ctx->d_seg_out.p, ctx->d_layer_out.p, ctx->stream), "combine");
+        ++ctx->launches;
+        if ((rc = read_back(ctx))) return rc;
+    }
+    (void)nseg;
     ctx->streaming = false;
     ctx->scored = true;
     ctx->pending = T > 0;

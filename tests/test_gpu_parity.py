@@ -536,7 +536,7 @@ def test_model_term_only(ampq, orc):
     fid, oid = _register(ampq, full, lts), _register(ampq, only, lts)
     full.score()
     only.score()
-    assert only.last_launch_count() == full.last_launch_count() - 1   # no amax launch
+    assert only.last_launch_count() == full.last_launch_count()   # a small scales launch stands in for the amax pass
     rng = np.random.default_rng(3)
     for a, b, lt in zip(fid, oid, lts):
         fr, orr = full.get_layer(a), only.get_layer(b)
