@@ -22,11 +22,13 @@ constexpr unsigned kSpinLimit = 1u << 22;  // polls of an mbarrier before a wait
 // A scoring tile (one partial sum per sample and accumulator) holds 2^shift
 // elements of a segment; the host picks the shift per score so that small
 // problems still spread over every SM and large ones pay few tile ends.
-constexpr int kMinTileShift = 15;
+constexpr int kMinTileShift = 13;
 constexpr int kMaxTileShift = 19;
 constexpr int kTileElems = 1 << kMaxTileShift;        // largest scoring tile
-constexpr int kAmaxTileElems = AMPQ_AMAX_TILE_ELEMS;  // elements of one amax tile
-static_assert((1 << kMinTileShift) % kSubElems == 0, "a scoring tile is a whole number of flush blocks");
+constexpr int kAmaxTileElems = AMPQ_AMAX_TILE_ELEMS;  // elements of one amax tile of a large pass
+constexpr int kMinAmaxTileElems = 4096;               // small passes take smaller tiles so that they still spread over the SMs
+static_assert(kSubElems % (1 << kMinTileShift) == 0, "a flush block is a whole number of the smallest scoring tiles");
+static_assert(kAmaxTileElems >= (1 << 15), "an amax tile holds whole rows of the largest triangular matrix");
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
 constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values

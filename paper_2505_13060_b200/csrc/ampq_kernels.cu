@@ -202,7 +202,7 @@ __global__ void resolve_amax_kernel(int T, const Tensor* __restrict__ tens, unsi
 }
 
 __global__ void __launch_bounds__(kThreads)
-amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T,
+amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_begin, int T, int tile_elems,
             unsigned* amax_bits, ScalesArgs tail) {
     __shared__ int s_slot;
     __shared__ int s_last;
@@ -210,9 +210,9 @@ amax_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile_
     const long long tile = blockIdx.x;
     const int t = find_tensor(tile_begin, T, tile, &s_slot);
     const Tensor& tn = tens[t];
-    const long long first = (tile - __ldg(tile_begin + t)) * (long long)kAmaxTileElems;
+    const long long first = (tile - __ldg(tile_begin + t)) * (long long)tile_elems;
     const long long left = tn.numel - first;
-    int n = left < kAmaxTileElems ? (int)left : kAmaxTileElems;
+    int n = left < tile_elems ? (int)left : tile_elems;
 #ifdef AMPQ_BOUNDS_CHECK
     if (first < 0 || left <= 0) n = 0;  // a tile outside its tensor is not read (the scoring pass reports it)
 #endif
@@ -1124,11 +1124,18 @@ cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, Lau
     return cudaGetLastError();
 }
 
-cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int tile_elems,
                         unsigned* amax_bits, cudaStream_t st, const ScalesArgs& tail) {
     if (ntiles <= 0) return cudaSuccess;
-    amax_kernel<<<(unsigned)ntiles, kThreads, 0, st>>>(tens, tile_begin, T, amax_bits, tail);
+    if (tile_elems < kMinAmaxTileElems || tile_elems > kAmaxTileElems) return cudaErrorInvalidValue;
+    amax_kernel<<<(unsigned)ntiles, kThreads, 0, st>>>(tens, tile_begin, T, tile_elems, amax_bits, tail);
     return cudaGetLastError();
+}
+
+int pick_amax_tile(long long elems, int sms) {
+    int tile = kAmaxTileElems;
+    while (tile > kMinAmaxTileElems && elems / tile < 4LL * sms) tile /= 2;
+    return tile;
 }
 
 cudaError_t launch_scales(int T, int fmask, const Tensor* tens, unsigned* amax_bits, float* scales, int* tensor_flags,

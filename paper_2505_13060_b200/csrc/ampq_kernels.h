@@ -39,8 +39,12 @@ struct CombineArgs {
 
 cudaError_t launch_init_amax(const Tensor* tens, int T, unsigned* amax_bits, LaunchStatus* status,
                              cudaStream_t st);
-cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles,
+// One CTA per tile of tile_elems elements (kMinAmaxTileElems..kAmaxTileElems; tile_begin counts such tiles).
+// Triangular operands need tile_elems = kAmaxTileElems (whole matrix rows per tile).
+cudaError_t launch_amax(const Tensor* tens, const long long* tile_begin, int T, long long ntiles, int tile_elems,
                         unsigned* amax_bits, cudaStream_t st, const ScalesArgs& tail = ScalesArgs());
+// Amax tile for a pass over `elems` elements on `sms` SMs: the largest that still gives every SM a few tiles.
+int pick_amax_tile(long long elems, int sms);
 // pow2 = 1: power-of-two scales instead of amax / fmax.  Tensors whose amax_src
 // names another tensor take (and record) that tensor's amax.
 cudaError_t launch_scales(int T, int fmask, const Tensor* tens, unsigned* amax_bits, float* scales, int* tensor_flags,

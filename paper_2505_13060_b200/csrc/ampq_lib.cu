@@ -120,6 +120,8 @@ struct ampq_ctx {
     int launches = 0;
     int max_ctas = kScoreCtasPerSm;  // persistent scoring grid: kScoreCtasPerSm CTAs per SM
     int tile_shift = kMaxTileShift;  // log2 of the scoring tile of the last score
+    int amax_tile = kAmaxTileElems;  // elements of an amax tile of the last pass
+    int sms = 1;
     std::string err;
 
     // tables of the last score (host copies)
@@ -237,16 +239,19 @@ int ensure_results(ampq_ctx* ctx, size_t T, size_t S, int nacc, size_t layer_dou
 // matrices, else 0 (scored densely, which gives the same sums).  The triangular
 // path needs a power-of-two T in [64, 32768], whole matrices per sample, and
 // 16-byte aligned sample slices of values and gradients.
-int causal_shift_of(const LayerRec& l, const Operand& o, const Tensor& t) {
+int causal_shift_of(const LayerRec& l, const Operand& o) {
     const long long T = o.causal_T;
     if (T <= 0 || !o.per_sample || (T & (T - 1))) return 0;
     int shift = 0;
     while ((1LL << shift) < T) ++shift;
     if (shift < kMinCausalShift || shift > kMaxCausalShift) return 0;
-    if (t.seg_len == 0 || t.seg_len % (T * T)) return 0;
+    const long long seg_len = extent_of(l, o);
+    if (seg_len == 0 || seg_len % (T * T)) return 0;
+    if (o.mem == AMPQ_MEM_HOST) return shift;  // staged: 256-byte aligned, samples back to back
     const int es = o.dtype == AMPQ_F32 ? 4 : 2;
-    if ((reinterpret_cast<uintptr_t>(t.values) & 15) || (reinterpret_cast<uintptr_t>(t.grads) & 15)) return 0;
-    if (l.R > 1 && (t.grad_stride * es) % 16) return 0;
+    if ((reinterpret_cast<uintptr_t>(o.values) & 15) || (reinterpret_cast<uintptr_t>(o.grads) & 15)) return 0;
+    if ((seg_len * es) % 16) return 0;
+    if (l.R > 1 && (o.grad_stride * es) % 16) return 0;
     return shift;
 }
 
@@ -318,6 +323,19 @@ int build_tables(ampq_ctx* ctx) {
         }
     }
     ctx->tile_shift = pick_tile_shift(scored_elems, ctx->max_ctas);
+    {   // amax tiles: smaller for a small pass; whole matrix rows per tile when a triangular operand is present
+        long long measured_elems = 0;
+        bool triangular = false;
+        for (const auto& l : ctx->layers) {
+            if (!layer_ready(l)) continue;
+            for (int k = 0; k < 2; ++k) {
+                if (l.op[k].amax_preset < 0.0f) measured_elems += l.op[k].numel;
+                triangular = triangular || causal_shift_of(l, l.op[k]) > 0;
+            }
+        }
+        ctx->amax_tile = triangular ? kAmaxTileElems : pick_amax_tile(measured_elems, ctx->sms);
+        if (triangular && ctx->tile_shift < kMaxCausalShift) ctx->tile_shift = kMaxCausalShift;  // a scoring tile holds whole rows too
+    }
     const long long tile_elems = 1LL << ctx->tile_shift;
     for (size_t li = 0; li < ctx->layers.size(); ++li) {
         LayerRec& l = ctx->layers[li];
@@ -365,7 +383,7 @@ int build_tables(ampq_ctx* ctx) {
                 t.gstream[j - 1] = reinterpret_cast<const char*>(t.grads) + (long long)j * t.grad_stride * es;
             t.seg_base = (int)ctx->segs.size();
             t.amax_preset = o.amax_preset;
-            t.causal_shift = causal_shift_of(l, o, t);
+            t.causal_shift = causal_shift_of(l, o);
             const int me = (int)ctx->tens.size();
             t.amax_src = me;
             const long long per_tensor_slots = (long long)l.R * t.tiles_per_seg;
@@ -378,7 +396,7 @@ int build_tables(ampq_ctx* ctx) {
             // first layer's tensor has one n-stream tile per (sample, value tile)
             long long my_tiles[kScoreClasses] = {};
             const int c0 = (o.dtype == AMPQ_F32 ? 0 : 1) * kMaxRB;  // classes of this operand's dtype
-            long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + kAmaxTileElems - 1) / kAmaxTileElems;
+            long long my_atiles = o.amax_preset >= 0.0f ? 0 : (o.numel + ctx->amax_tile - 1) / ctx->amax_tile;
             if (grp && pos > 0) {
                 t.share_n = 0;
                 t.partial_base = grp->leader_base + pos * per_tensor_slots;
@@ -636,12 +654,13 @@ int ensure_job_partials(ampq_ctx* ctx, size_t n) {
 int job_amax_and_scales(ampq_ctx* ctx, SegmentJob* job, LaunchStatus* status, int dtype, const void* values,
                         const void* grads, long long numel, float preset, long long ntiles) {
     cudaStream_t st = ctx->stream;
-    const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
+    const int atile = pick_amax_tile(numel, ctx->sms);
+    const long long namax = preset >= 0.0f ? 0 : (numel + atile - 1) / atile;
     // with a preset the scales are formed while the tables are filled; otherwise by the last CTA of the amax pass
     AMPQ_CUDA(launch_job_prepare(job, values, grads, numel, dtype, preset, ntiles, namax, ctx->fmask, ctx->scale_pow2, status, st), "job_prepare");
     ++ctx->launches;
     if (namax > 0) {
-        AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, &job->amax_bits, st,
+        AMPQ_CUDA(launch_amax(&job->tensor, job->amax_tile_begin, 1, namax, atile, &job->amax_bits, st,
                               scales_args(1, ctx->fmask, &job->tensor, &job->amax_bits, job->scales, &job->flag, status,
                                           ctx->scale_pow2, &job->amax_done)), "amax");
         ++ctx->launches;
@@ -690,6 +709,7 @@ int ampq_create(ampq_ctx** out, int device, void* cuda_stream) {
         return AMPQ_ERR_CUDA;
     }
     ctx->max_ctas = kScoreCtasPerSm * sms;
+    ctx->sms = sms;
     *out = ctx;
     return AMPQ_OK;
 }
@@ -821,7 +841,7 @@ int ampq_measure_amax(ampq_ctx* ctx) {
     if ((rc = stage_host_operands(ctx))) return rc;
     if (T > 0) {
         AMPQ_CUDA(launch_init_amax(ctx->d_tens.p, T, ctx->d_amax_bits.p, ctx->d_status.p, st), "init_amax");
-        AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st), "amax");
+        AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->amax_tile, ctx->d_amax_bits.p, st), "amax");
         ctx->launches = ctx->namax_tiles > 0 ? 2 : 1;
         if (ctx->n_amax_alias > 0) {
             AMPQ_CUDA(launch_resolve_amax(T, ctx->d_tens.p, ctx->d_amax_bits.p, st), "resolve_amax");
@@ -884,7 +904,7 @@ int ampq_score(ampq_ctx* ctx) {
                                           ctx->d_status.p, ctx->scale_pow2, &ctx->d_status.p->amax_done);
         const bool amax_pass = ctx->namax_tiles > 0 && ctx->measured;
         if (amax_pass) {
-            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->d_amax_bits.p, st, sa), "amax");
+            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->amax_tile, ctx->d_amax_bits.p, st, sa), "amax");
             ++ctx->launches;
         }
         if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched

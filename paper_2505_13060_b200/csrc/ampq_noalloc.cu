@@ -161,7 +161,7 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     noalloc_prepare_kernel<<<1, 32, 0, st>>>(s, values, grads, numel, dtype, preset, ntiles, namax);
     bool ok = cudaGetLastError() == cudaSuccess;
     ok = ok && launch_init_amax(&s->tensor, 1, &s->amax_bits, &s->status, st) == cudaSuccess;
-    ok = ok && launch_amax(&s->tensor, s->amax_tile_begin, 1, namax, &s->amax_bits, st) == cudaSuccess;
+    ok = ok && launch_amax(&s->tensor, s->amax_tile_begin, 1, namax, kAmaxTileElems, &s->amax_bits, st) == cudaSuccess;
     ok = ok && launch_scales(1, fmask, &s->tensor, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
     int sms = 0;
     ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;

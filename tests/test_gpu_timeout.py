@@ -24,14 +24,14 @@ def _tensors():
     import torch
 
     g = torch.Generator(device="cuda").manual_seed(33)
-    n = 8 * 1024 * 1024   # 16-byte aligned bf16: every chunk goes through the ring
+    n = 128 * 1024 * 1024   # 16-byte aligned bf16, far larger than L2: the scoring warps keep catching up with HBM
     v = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1, generator=g)
     gr = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3, generator=g)
     return v, gr
 
 
-def _bind(ampq, ctx, lid, v, gr, offset):
-    n = v.numel() - 8
+def _bind(ampq, ctx, lid, v, gr, offset, n=None):
+    n = n or v.numel() - 8
     es = v.element_size()
     ctx.bind_operand(lid, 0, ampq.BF16, v.data_ptr() + offset * es, n, True, gr.data_ptr() + offset * es, n)
     ctx.bind_operand(lid, 1, ampq.BF16, 0, 0, False, 0, 0)
@@ -60,7 +60,7 @@ def worker():
     assert ampq.lib().ampq_get_operand(ctx._h, lid, 0, np.zeros(2).ctypes.data) == ampq.ERR_TIMEOUT
     torch.cuda.synchronize()   # the device is fine: no error is pending
     # the same context, same tensors one element off the 16-byte grid: nothing goes through the ring
-    n = _bind(ampq, ctx, lid, v, gr, 1)
+    n = _bind(ampq, ctx, lid, v, gr, 1, 4 * 1024 * 1024)
     ctx.score()
     got = ctx.get_operand(lid, 0)[0]
     a, _, _, seg = orc.score_operand(synth.to_numpy(v)[1:1 + n].reshape(1, -1), synth.to_numpy(gr)[1:1 + n].reshape(1, -1),
@@ -85,7 +85,7 @@ def test_stage_wait_that_runs_out_is_reported_and_leaves_the_context_usable(tmp_
     ctx = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
     ctx.set_formats([0, 1])
     lid = ctx.register_layer(ampq.LINEAR, "ring", 1)
-    n = _bind(ampq, ctx, lid, v, gr, 0)
+    n = _bind(ampq, ctx, lid, v, gr, 0, 16 * 1024 * 1024)
     ctx.score()
     got = ctx.get_operand(lid, 0)[0]
     _, _, _, seg = orc.score_operand(synth.to_numpy(v)[:n].reshape(1, -1), synth.to_numpy(gr)[:n].reshape(1, -1), 1, True, [1])
