@@ -23,7 +23,10 @@ constexpr unsigned kSpinLimit = 1u << 22;  // polls of an mbarrier before a wait
 // elements of a segment; the host picks the shift per score so that small
 // problems still spread over every SM and large ones pay few tile ends.
 constexpr int kMinTileShift = 13;
-constexpr int kMaxTileShift = 19;
+#ifndef AMPQ_MAX_TILE_SHIFT
+#define AMPQ_MAX_TILE_SHIFT 21
+#endif
+constexpr int kMaxTileShift = AMPQ_MAX_TILE_SHIFT;
 constexpr int kTileElems = 1 << kMaxTileShift;        // largest scoring tile
 constexpr int kAmaxTileElems = AMPQ_AMAX_TILE_ELEMS;  // elements of one amax tile of a large pass
 constexpr int kMinAmaxTileElems = 4096;               // small passes take smaller tiles so that they still spread over the SMs

@@ -902,15 +902,18 @@ int ampq_score(ampq_ctx* ctx) {
         // nothing is measured, by a small launch of their own
         const ScalesArgs sa = scales_args(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p,
                                           ctx->d_status.p, ctx->scale_pow2, &ctx->d_status.p->amax_done);
+        // (the tail costs every amax CTA one atomic on a single word: only worth it for a small pass)
         const bool amax_pass = ctx->namax_tiles > 0 && ctx->measured;
+        const bool tail = amax_pass && ctx->namax_tiles <= 4096;
         if (amax_pass) {
-            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->amax_tile, ctx->d_amax_bits.p, st, sa), "amax");
+            AMPQ_CUDA(launch_amax(ctx->d_tens.p, ctx->d_amax_tile_begin.p, T, ctx->namax_tiles, ctx->amax_tile, ctx->d_amax_bits.p, st,
+                                  tail ? sa : ScalesArgs()), "amax");
             ++ctx->launches;
         }
         if (!ctx->measured && ctx->nslots > 0)  // the S-only kernels leave the D columns of a slot untouched
             AMPQ_CUDA(cudaMemsetAsync(ctx->d_partials.p, 0, (size_t)ctx->nslots * nacc * sizeof(double), st), "memset partials");
         if (tm) AMPQ_CUDA(cudaEventRecord(ctx->ev[2], st), "cudaEventRecord");
-        if (!amax_pass) {
+        if (!tail) {
             AMPQ_CUDA(launch_scales(T, ctx->fmask, ctx->d_tens.p, ctx->d_amax_bits.p, ctx->d_scales.p, ctx->d_flags.p, ctx->d_status.p, st, ctx->scale_pow2), "scales");
             ++ctx->launches;
         }

@@ -27,8 +27,8 @@
 namespace ampq {
 namespace {
 
-constexpr long long kNoAllocMaxTiles = AMPQ_NOALLOC_MAX_NUMEL / kTileElems;
-static_assert(AMPQ_NOALLOC_MAX_NUMEL % kTileElems == 0, "the size limit is a whole number of scoring tiles");
+constexpr long long kNoAllocMaxTiles = 4096;  // per-tile partial slots in the fixed array
+static_assert(AMPQ_NOALLOC_MAX_NUMEL <= kNoAllocMaxTiles * (long long)kTileElems, "the largest segment fits in the slots at the largest tile");
 constexpr int kNoAllocAcc = 2;  // S and D of the one low-precision format
 constexpr int kMaxDevices = 64;
 
@@ -155,7 +155,12 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     const float preset = amax > 0.0f ? amax : (amax == 0.0f ? 0.0f : -1.0f);  // -0 -> +0
-    const long long ntiles = (numel + kTileElems - 1) / kTileElems;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) { cudaGetLastError(); return AMPQ_ERR_CUDA; }
+    // the tile the ordinary pass would take for this size, enlarged until the tiles fit in the fixed slots
+    int shift = pick_tile_shift(numel, kScoreCtasPerSm * sms);
+    while (shift < kMaxTileShift && ((numel + (1LL << shift) - 1) >> shift) > kNoAllocMaxTiles) ++shift;
+    const long long ntiles = (numel + (1LL << shift) - 1) >> shift;
     const long long namax = preset >= 0.0f ? 0 : (numel + kAmaxTileElems - 1) / kAmaxTileElems;
     const int fmask = fmt == AMPQ_FMT_E4M3 ? kMaskE4M3 : kMaskE5M2;
     noalloc_prepare_kernel<<<1, 32, 0, st>>>(s, values, grads, numel, dtype, preset, ntiles, namax);
@@ -163,9 +168,7 @@ int ampq_score_segment_noalloc(int device, void* cuda_stream, int dtype, int fmt
     ok = ok && launch_init_amax(&s->tensor, 1, &s->amax_bits, &s->status, st) == cudaSuccess;
     ok = ok && launch_amax(&s->tensor, s->amax_tile_begin, 1, namax, kAmaxTileElems, &s->amax_bits, st) == cudaSuccess;
     ok = ok && launch_scales(1, fmask, &s->tensor, &s->amax_bits, s->scales, &s->flag, &s->status, st) == cudaSuccess;
-    int sms = 0;
-    ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
-    ok = ok && launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &s->tensor, s->tile_begin, 1, ntiles, kMaxTileShift, kScoreCtasPerSm * sms, fmask, s->scales,
+    ok = ok && launch_score(dtype == AMPQ_F32 ? 0 : 1, 1, &s->tensor, s->tile_begin, 1, ntiles, shift, kScoreCtasPerSm * sms, fmask, s->scales,
                             s->partials, &s->status, st) == cudaSuccess;
     ok = ok && launch_finalize(&s->segment, 1, kNoAllocAcc, s->partials, s->seg_out, st) == cudaSuccess;
     if (ok) {
