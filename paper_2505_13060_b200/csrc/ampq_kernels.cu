@@ -1151,9 +1151,12 @@ cudaError_t launch_resolve_amax(int T, const Tensor* tens, unsigned* amax_bits, 
     return cudaGetLastError();
 }
 
+#ifndef AMPQ_TILES_PER_CTA
+#define AMPQ_TILES_PER_CTA 16   // tiles a CTA of the persistent grid should get before tiles stop shrinking
+#endif
 int pick_tile_shift(long long scored_elems, int max_ctas) {
     int shift = kMaxTileShift;
-    while (shift > kMinTileShift && (scored_elems >> shift) < 48LL * max_ctas) --shift;
+    while (shift > kMinTileShift && (scored_elems >> shift) < (long long)AMPQ_TILES_PER_CTA * max_ctas) --shift;
     return shift;
 }
 

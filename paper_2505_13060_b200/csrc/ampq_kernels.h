@@ -70,7 +70,7 @@ cudaError_t launch_score(int dtype, int rb, const Tensor* tens, const long long*
                          int tile_shift, int max_ctas, int fmask, const float* scales, double* partials,
                          LaunchStatus* status, cudaStream_t st, int causal = 0, int out_stride = 0);
 // Largest tile shift in [kMinTileShift, kMaxTileShift] that still gives a grid of
-// max_ctas CTAs a few dozen tiles each (or the smallest shift when even that does not).
+// max_ctas CTAs 16 tiles each (or the smallest shift when even that does not).
 int pick_tile_shift(long long scored_elems, int max_ctas);
 cudaError_t launch_finalize(const Segment* segs, int nseg, int nacc, const double* partials, double* seg_out,
                             cudaStream_t st, const CombineArgs& tail = CombineArgs());
