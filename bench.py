@@ -397,7 +397,7 @@ def run_b200(args):
         ctx.score()
         t = ctx.get_timing()  # synchronises the step; the per-kernel events are the library's own
         if shard_layers:
-            rows = {g: shard.layer_row(ctx.get_layer(lid), F) for g, lid in zip(my_global, ids)}
+            rows = dict(zip(my_global, ctx.get_layer_table(ids)))
             table = shard.gather_layer_table(rows, n_layers_model, F, device=dev)
             all_low = float(table[:, 1 + F + 1].sum())
             plan = shard.select_from_table(ampq, table, F, groups, ampq.D_MEASURED, 0.2 * all_low)
@@ -548,19 +548,25 @@ def run_b200(args):
             # every byte the step reads on rank 0 (the amax pass reads each operand once more)
             "whole_pass_traffic": {"bytes_read_per_gpu": read_bytes, "gbs": whole_gbs, "frac_of_measured_peak": whole_gbs / peak},
         }
-        # A step cannot read HBM much faster than the measured copy peak: such a
-        # number means the timed region skipped work, so it is not reported.
-        limit = 1.2 * peak
-        too_fast = [k for k, v in (("whole_pass_traffic.gbs", whole_gbs), ("roofline.amax_kernel_gbs", roofline["amax_kernel_gbs"]),
-                                   ("roofline.achieved (bytes read)", pass_bytes["score"] / (k_ms * 1e-3) / 1e9))
-                    if v is not None and v > limit]
-        if too_fast:
-            line["rejected_value"] = value
-            line["value"] = None
-            line["invalid"] = "implausible: %s above 1.2 x the measured HBM peak (%.0f GB/s)" % (", ".join(too_fast), limit)
+        reject_implausible(line, peak, {"whole_pass_traffic.gbs": whole_gbs,
+                                        "roofline.amax_kernel_gbs": roofline["amax_kernel_gbs"],
+                                        "scoring launches (bytes read / kernel time)": pass_bytes["score"] / (k_ms * 1e-3) / 1e9})
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def reject_implausible(line: dict, peak_gbs: float, rates: dict) -> bool:
+    """A step cannot read HBM much faster than the measured copy peak: a byte rate
+    above 1.2 x that peak means the timed region skipped work, and the line then
+    carries ``value: null`` with the reason instead of a number."""
+    limit = 1.2 * peak_gbs
+    too_fast = [k for k, v in rates.items() if v is not None and v > limit]
+    if too_fast:
+        line["rejected_value"] = line["value"]
+        line["value"] = None
+        line["invalid"] = "implausible: %s above 1.2 x the measured HBM peak (%.0f GB/s)" % (", ".join(too_fast), limit)
+    return bool(too_fast)
 
 
 def relaunch_ranks(args):

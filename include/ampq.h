@@ -251,6 +251,13 @@ int ampq_get_layer(ampq_ctx *ctx, int layer_id, float *amax, float *scale, float
                    double *s_per_sample, double *s_mean, double *d_meas_per_sample,
                    double *d_model, double *d_meas);
 
+/* The per-layer table of n layers in one call (synchronises like ampq_get_layer):
+ * out is [n][1 + 2F] row-major, row i = {s_l, d_model[0..F-1], d_meas[0..F-1]} of
+ * layer layer_ids[i] -- what the sub-graph sums and the selection need, and what
+ * processes that share a model exchange.  Host pointers.  AMPQ_ERR_NONFINITE
+ * (rows still written) if one of the layers held Inf/NaN. */
+int ampq_get_layer_table(ampq_ctx *ctx, const int *layer_ids, int n, double *out);
+
 /* Per-operand sums of a layer: out[R*F], index r*F + a, a = 0: S, a = f >= 1:
  * D_f.  Host pointer. */
 int ampq_get_operand(ampq_ctx *ctx, int layer_id, int operand, double *out);

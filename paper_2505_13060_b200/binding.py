@@ -38,7 +38,7 @@ EXPORTS = [
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
     "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal", "ampq_set_measured",
-    "ampq_set_sharing", "ampq_get_pass_bytes", "ampq_merge_sample_tables",
+    "ampq_set_sharing", "ampq_get_pass_bytes", "ampq_merge_sample_tables", "ampq_get_layer_table",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -79,6 +79,7 @@ def lib():
     L.ampq_get_timing.argtypes = [vp, fp]
     L.ampq_get_layer.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, vp, vp]
     L.ampq_get_operand.argtypes = [vp, i, i, vp]
+    L.ampq_get_layer_table.argtypes = [vp, vp, i, vp]
     L.ampq_export_codes.argtypes = [vp, i, i, i, vp]
     L.ampq_define_group.argtypes = [vp, vp, i, vp, vp, i, ip]
     L.ampq_clear_groups.argtypes = [vp]
@@ -355,6 +356,13 @@ class Context:
         return dict(amax=amax, scale=scale.reshape(2, F), inv_scale=inv.reshape(2, F), s_per_sample=s_r,
                     s_mean=float(s_mean[0]), d_meas_per_sample=d_meas_r.reshape(R, F), d_model=d_model,
                     d_meas=d_meas, status=rc)
+
+    def get_layer_table(self, layer_ids) -> np.ndarray:
+        """[n, 1 + 2F] rows {s_mean, d_model[F], d_meas[F]} of the given layers, one call."""
+        ids = np.ascontiguousarray(layer_ids, dtype=np.int32)
+        out = np.zeros((ids.size, 1 + 2 * self.F))
+        self._check(lib().ampq_get_layer_table(self._h, _np_ptr(ids), ids.size, _np_ptr(out)))
+        return out
 
     def get_operand(self, layer_id: int, operand: int) -> np.ndarray:
         out = np.zeros((self._R[layer_id], self.F))

@@ -1174,6 +1174,28 @@ int ampq_get_layer(ampq_ctx* ctx, int layer_id, float* amax, float* scale, float
     return AMPQ_OK;
 }
 
+int ampq_get_layer_table(ampq_ctx* ctx, const int* layer_ids, int n, double* out) {
+    if (!ctx || n < 0 || (n > 0 && (!layer_ids || !out))) return AMPQ_ERR_INVALID;
+    DeviceGuard g(ctx->device);
+    int rc = sync_results(ctx);
+    if (rc) return rc;
+    const int F = ctx->F, K = 1 + 2 * F;
+    bool bad = false;
+    for (int i = 0; i < n; ++i) {
+        if ((rc = check_layer(ctx, layer_ids[i]))) return rc;
+        const LayerRec& l = ctx->layers[layer_ids[i]];
+        if (l.scored < 0) return fail(ctx, AMPQ_ERR_STATE, "layer '" + l.name + "' was not part of the last score");
+        const Layer& ly = ctx->lay[l.scored];
+        bad = bad || ctx->h_flags.p[ly.tensor0] != 0 || ctx->h_flags.p[ly.tensor1] != 0;
+        const double* o = layer_block(ctx, l.scored);
+        double* row = out + (size_t)i * K;
+        row[0] = o[ly.R];
+        std::memcpy(row + 1, o + ly.R + 1 + (long long)ly.R * F, sizeof(double) * 2 * F);  // d_model[F], d_meas[F]
+    }
+    if (bad) return fail(ctx, AMPQ_ERR_NONFINITE, "a layer of the table holds Inf/NaN");
+    return AMPQ_OK;
+}
+
 int ampq_get_operand(ampq_ctx* ctx, int layer_id, int operand, double* out) {
     int rc = check_layer(ctx, layer_id);
     if (rc) return rc;

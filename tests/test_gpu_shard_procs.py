@@ -49,6 +49,8 @@ def _score(which):
         binding.bind_layer_tensors(ctx, ids[i], lt)
     ctx.score()
     rows = {i: shard.layer_row(ctx.get_layer(lid), F) for i, lid in ids.items()}
+    bulk = ctx.get_layer_table(list(ids.values()))   # the same rows in one call
+    assert all(np.array_equal(bulk[k], rows[i]) for k, i in enumerate(ids))
     ctx.destroy()
     return rows
 
