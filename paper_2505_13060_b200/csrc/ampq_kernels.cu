@@ -22,6 +22,7 @@
 #include <cuda_fp16.h>
 #include <atomic>
 #include <cstdint>
+#include <type_traits>
 
 #include "ampq_device.h"
 #include "ampq_kernels.h"
@@ -512,8 +513,8 @@ struct RingPos {
 // thread a < RB*NACC writes partial (r, a) of the tile.  s_red holds one
 // kConsumers/32 x RB*NACC block; the caller alternates two blocks from tile to
 // tile so that a tile's readers never meet the next tile's writers.
-template <int NACC, int RB>
-__device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], double* s_red,
+template <int NACC, int RB, class A64>
+__device__ __forceinline__ void reduce_and_store(const A64& acc, double* s_red,
                                                  double* __restrict__ partials, long long slot0,
                                                  long long slot_stride, int out_stride) {
     constexpr int NV = RB * NACC;
@@ -522,7 +523,7 @@ __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], 
     for (int r = 0; r < RB; ++r) {
 #pragma unroll
         for (int a = 0; a < NACC; ++a) {
-            double x = acc[r][a];
+            double x = acc.get(r, a);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
             if (lane == 0) s_red[warp * NV + r * NACC + a] = x;
@@ -538,13 +539,47 @@ __device__ __forceinline__ void reduce_and_store(const double (&acc)[RB][NACC], 
     }
 }
 
+// The fp64 accumulators of a tile, one set per scoring thread: in registers, or,
+// with three and four gradient streams, where the registers run out, in this
+// thread's column of a shared-memory block (entry (r, a) of thread t at
+// [(r * NACC + a) * kConsumers + t]: consecutive threads, consecutive words).
 template <int NACC, int RB>
-__device__ __forceinline__ void flush_acc(Acc<NACC> (&acc)[RB], double (&acc64)[RB][NACC]) {
+struct Acc64Reg {
+    double v[RB][NACC];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) v[r][a] = 0.0;
+    }
+    __device__ __forceinline__ void add(int r, int a, double x) { v[r][a] += x; }
+    __device__ __forceinline__ double get(int r, int a) const { return v[r][a]; }
+};
+template <int NACC, int RB>
+struct Acc64Smem {
+    double* col;
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int k = 0; k < RB * NACC; ++k) col[k * kConsumers] = 0.0;
+    }
+    __device__ __forceinline__ void add(int r, int a, double x) { col[(r * NACC + a) * kConsumers] += x; }
+    __device__ __forceinline__ double get(int r, int a) const { return col[(r * NACC + a) * kConsumers]; }
+};
+#ifndef AMPQ_ACC64_SMEM_FROM
+#define AMPQ_ACC64_SMEM_FROM 3   // gradient streams from which the fp64 accumulators live in shared memory
+#endif
+template <int RB>
+constexpr bool kAcc64InSmem = RB >= AMPQ_ACC64_SMEM_FROM;
+template <int NACC, int RB>
+using Acc64 = typename std::conditional<kAcc64InSmem<RB>, Acc64Smem<NACC, RB>, Acc64Reg<NACC, RB>>::type;
+
+template <int NACC, int RB, class A64>
+__device__ __forceinline__ void flush_acc(Acc<NACC> (&acc)[RB], A64& acc64) {
 #pragma unroll
     for (int r = 0; r < RB; ++r)
 #pragma unroll
         for (int a = 0; a < NACC; ++a) {
-            acc64[r][a] += (double)acc[r].v[a].x + (double)acc[r].v[a].y;
+            acc64.add(r, a, (double)acc[r].v[a].x + (double)acc[r].v[a].y);
             acc[r].v[a] = make_float2(0.0f, 0.0f);
         }
 }
@@ -552,10 +587,9 @@ __device__ __forceinline__ void flush_acc(Acc<NACC> (&acc)[RB], double (&acc64)[
 // n elements straight from global memory (what the ring does not carry: ragged
 // ends and tensors that are not 16-byte aligned), in blocks of kSubElems so that
 // an fp32 accumulator lane never sees more than kSubElems / kConsumers terms.
-template <int DT, int FMASK, int RB>
+template <int DT, int FMASK, int RB, class A64>
 __device__ __forceinline__ void score_direct(const char* vbase, const char* const (&gbase)[RB], int n,
-                                             const float2 (&inv2)[2], const float2 (&nsc2)[2],
-                                             double (&acc64)[RB][Fm<FMASK>::kAcc]) {
+                                             const float2 (&inv2)[2], const float2 (&nsc2)[2], A64& acc64) {
     constexpr int NACC = Fm<FMASK>::kAcc;
     const int es = Elem<DT>::kBytes;
     for (int sub = 0; sub < n; sub += kSubElems) {
@@ -582,7 +616,7 @@ __device__ __forceinline__ void score_direct(const char* vbase, const char* cons
 template <int DT, int FMASK>
 __device__ __forceinline__ void score_causal_rows(const char* vbase, const char* gbase, int n, long long row0,
                                                   int shift, const float2 (&inv2)[2], const float2 (&nsc2)[2],
-                                                  double (&acc64)[1][Fm<FMASK>::kAcc]) {
+                                                  Acc64Reg<Fm<FMASK>::kAcc, 1>& acc64) {
     using E = Elem<DT>;
     constexpr int NACC = Fm<FMASK>::kAcc;
     constexpr int NP = E::kPerVec / 2;
@@ -647,18 +681,19 @@ struct Ring {
     static_assert(kStages >= 2, "the ring needs at least two stages");
     static constexpr int kRingBytes = kStages * kStageBytes;
     static constexpr int kRedDoubles = 2 * (kConsumers / 32) * RB * kMaxAcc;
-    // ring | full[kStages] empty[kStages] | reduction blocks | abort flag
-    static constexpr int kSmemBytes = kRingBytes + 2 * kStages * 8 + kRedDoubles * 8 + 16;
+    static constexpr int kAcc64Doubles = kAcc64InSmem<RB> ? RB * kMaxAcc * kConsumers : 0;  // fp64 accumulators kept in shared memory
+    // ring | full[kStages] empty[kStages] | reduction blocks | fp64 accumulators | abort flag
+    static constexpr int kSmemBytes = kRingBytes + 2 * kStages * 8 + (kRedDoubles + kAcc64Doubles) * 8 + 16;
 };
 
 // The scoring warps' side of the ring for one tile: nchunks stages, each
 // taken into registers, handed back, then scored.
-template <int DT, int FMASK, int RB>
+template <int DT, int FMASK, int RB, class A64>
 __device__ __forceinline__ void consume_chunks(int nchunks, const unsigned char* ring, unsigned long long* full,
                                                unsigned long long* empty, RingPos<Ring<RB>::kStages>& pos,
                                                volatile int* s_abort, const float2 (&inv2)[2],
                                                const float2 (&nsc2)[2], Acc<Fm<FMASK>::kAcc> (&acc)[RB],
-                                               double (&acc64)[RB][Fm<FMASK>::kAcc]) {
+                                               A64& acc64) {
     using RG = Ring<RB>;
     using E = Elem<DT>;
     constexpr int NACC = Fm<FMASK>::kAcc;
@@ -782,7 +817,8 @@ __device__ __forceinline__ void score_tiles(const Tensor* __restrict__ tens, con
                                             long long ntiles, int tile_shift, const float* __restrict__ scales,
                                             double* __restrict__ partials, LaunchStatus* __restrict__ status,
                                             int out_stride, const unsigned char* ring, unsigned long long* full,
-                                            unsigned long long* empty, double* s_red, volatile int* s_abort) {
+                                            unsigned long long* empty, double* s_red, double* s_acc64,
+                                            volatile int* s_abort) {
     using RG = Ring<RB>;
     constexpr int NACC = Fm<FMASK>::kAcc;
     RingPos<RG::kStages> pos;  // the same walk of the ring as the producer's
@@ -814,15 +850,14 @@ __device__ __forceinline__ void score_tiles(const Tensor* __restrict__ tens, con
         }
         const int nchunks = aligned && !CAUSAL ? (int)(((long long)q.n * es) / RG::kChunkBytes) : 0;
 
-        double acc64[RB][NACC];
+        Acc64<NACC, RB> acc64;
+        if constexpr (kAcc64InSmem<RB>) acc64.col = s_acc64 + threadIdx.x;
+        acc64.zero();
         Acc<NACC> acc[RB];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
-            for (int a = 0; a < NACC; ++a) {
-                acc64[r][a] = 0.0;
-                acc[r].v[a] = make_float2(0.0f, 0.0f);
-            }
+            for (int a = 0; a < NACC; ++a) acc[r].v[a] = make_float2(0.0f, 0.0f);
         consume_chunks<DT, FMASK, RB>(nchunks, ring, full, empty, pos, s_abort, inv2, nsc2, acc, acc64);
         flush_acc<NACC, RB>(acc, acc64);
         // what the ring did not carry
@@ -868,7 +903,8 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
     unsigned long long* full = reinterpret_cast<unsigned long long*>(smem + RG::kRingBytes);
     unsigned long long* empty = full + RG::kStages;
     double* s_red = reinterpret_cast<double*>(empty + RG::kStages);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(s_red + RG::kRedDoubles);
+    double* s_acc64 = s_red + RG::kRedDoubles;
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_acc64 + RG::kAcc64Doubles);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < RG::kStages; ++s) {
@@ -916,7 +952,7 @@ score_kernel(const Tensor* __restrict__ tens, const long long* __restrict__ tile
         }
     } else {
         score_tiles<DT, FMASK, RB, CAUSAL>(tens, tile_begin, ntiles, tile_shift, scales, partials, status, out_stride,
-                                           ring, full, empty, s_red, s_abort);
+                                           ring, full, empty, s_red, s_acc64, s_abort);
     }
     // Every thread of the CTA meets here: the producer has stopped issuing and the
     // scoring warps have stopped taking stages.  If a wait ran out on either side,
