@@ -611,8 +611,11 @@ __device__ __forceinline__ void score_direct(const char* vbase, const char* cons
 // which only the vectors on or left of the diagonal are read -- straight from
 // global memory, because a row's kept part is one short contiguous run and the
 // ring would need one bulk copy per row and stream (the copy rate, not the
-// bytes, then sets the pace).  Warp w takes rows w, w + 8, ... of the tile;
-// its lanes stride over the row's vectors with kU loads per stream in flight.
+// bytes, then sets the pace).  A warp takes groups of consecutive rows (groups
+// strided over the warps).  Its work items are (row, slot of 32 vectors); every
+// lane keeps kU items per stream in flight, and the items run on from one row
+// of the group into the next, so that a short row, or the ragged end of a long
+// one, leaves at most 31 lanes of one item idle instead of most of kU items.
 template <int DT, int FMASK>
 __device__ __forceinline__ void score_causal_rows(const char* vbase, const char* gbase, int n, long long row0,
                                                   int shift, const float2 (&inv2)[2], const float2 (&nsc2)[2],
@@ -621,23 +624,35 @@ __device__ __forceinline__ void score_causal_rows(const char* vbase, const char*
     constexpr int NACC = Fm<FMASK>::kAcc;
     constexpr int NP = E::kPerVec / 2;
     constexpr int kU = 4;
+    constexpr int kWarps = kConsumers / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nrows = n >> shift;
+    // rows per group: up to 8, fewer when the tile has too few rows to give every warp a group
+    int group = nrows / kWarps;
+    group = group < 1 ? 1 : (group > 8 ? 8 : group);
     Acc<NACC> acc[1];
 #pragma unroll
     for (int a = 0; a < NACC; ++a) acc[0].v[a] = make_float2(0.0f, 0.0f);
     int since_flush = 0;
-    for (int r = warp; r < nrows; r += kConsumers / 32) {
-        const int nv = causal_row_vectors(row0 + r, shift, E::kPerVec);
-        const uint4* vp = reinterpret_cast<const uint4*>(vbase + ((long long)r << shift) * E::kBytes);
-        const uint4* gp = reinterpret_cast<const uint4*>(gbase + ((long long)r << shift) * E::kBytes);
-        for (int c = lane; c < nv; c += 32 * kU) {
+    for (int r0 = warp * group; r0 < nrows; r0 += kWarps * group) {
+        const int r1 = r0 + group < nrows ? r0 + group : nrows;
+        int r = r0;                                                     // the next item: row r, vectors c .. c + 31
+        int c = 0;
+        int nv = causal_row_vectors(row0 + r, shift, E::kPerVec);
+        while (r < r1) {
             uint4 v[kU], g[kU];
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
-                const bool live = c + 32 * u < nv;
-                v[u] = live ? ld_stream_v4(vp + c + 32 * u) : make_uint4(0, 0, 0, 0);
-                g[u] = live ? ld_stream_v4(gp + c + 32 * u) : make_uint4(0, 0, 0, 0);
+                const bool live = r < r1 && c + lane < nv;
+                const long long off = (((long long)r << shift) * E::kBytes) + (long long)(c + lane) * 16;
+                v[u] = live ? ld_stream_v4(vbase + off) : make_uint4(0, 0, 0, 0);
+                g[u] = live ? ld_stream_v4(gbase + off) : make_uint4(0, 0, 0, 0);
+                c += 32;
+                if (r < r1 && c >= nv) {  // on to the next row of the group (uniform over the warp)
+                    ++r;
+                    c = 0;
+                    if (r < r1) nv = causal_row_vectors(row0 + r, shift, E::kPerVec);
+                }
             }
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
