@@ -52,8 +52,8 @@ FALLBACK_HBM_GBS = 6650.0
 # source it was taken on: `kernels_sha256` is the digest of ampq_kernels.cu +
 # ampq_device.h at capture time, and the bench reports traffic = null otherwise.
 NCU_TRAFFIC = {
-    "kernels_sha256": "88cc1544e4c4719dd36c71608d983503dbcfb9bbc4b3c9fa5aef2c8472e8e3dd",
-    "dram_bytes_per_scored_byte": {"e4m3": 1.0063},
+    "kernels_sha256": "ea299ed6543589acb49cb11c0459c9ebf8cd53602acade7586932a4abb893071",
+    "dram_bytes_per_scored_byte": {"e4m3": 1.0061},
     "source": "profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md",
 }
 
