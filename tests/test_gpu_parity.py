@@ -262,6 +262,12 @@ def test_preset_amax_saturates(ampq, orc):
     ctx.set_amax(lid, 0, -1.0)  # back to the measured amax
     ctx.score()
     compare_layer(ampq, ctx, lid, oracle_layer(orc, lt, [E4M3]), 2, "measured again")
+    # a preset of minus zero is a preset of zero (neutral scales), not a non-finite amax
+    ctx.set_amax(lid, 0, -0.0)
+    ctx.score()
+    got = ctx.get_layer(lid)
+    assert got["status"] == 0 and got["amax"][0].tobytes() == np.float32(0.0).tobytes()
+    assert got["scale"][0, 1] == 1.0 and got["inv_scale"][0, 1] == 1.0
     ctx.destroy()
 
 

@@ -37,6 +37,12 @@ def test_streamed_samples_match_oracle_and_full_score(ampq, orc, dtype):
     for lid, a in zip(ids, amax_x):
         ctx.set_amax(lid, 0, a)
     ctx.stream_begin()
+    # settings that shape the results cannot change under a streaming pass
+    L = ampq.lib()
+    fm = (__import__("ctypes").c_int * 2)(0, E5M2)
+    assert L.ampq_set_formats(ctx._h, fm, 2) == ampq.ERR_STATE
+    assert L.ampq_set_scale_mode(ctx._h, ampq.SCALE_POW2) == ampq.ERR_STATE
+    assert L.ampq_set_measured(ctx._h, 0) == ampq.ERR_STATE
     for r in range(R):   # samples arrive one at a time, layers in any order
         for lid, lt in reversed(list(zip(ids, lts))):
             x, gx = lt.values[0][r], lt.grads[0][r]

@@ -126,6 +126,30 @@ def test_select_matches_plain_branch_and_bound(ampq, orc, J, P, fracs):
         assert got[0].tolist() == ref[0].tolist() and got[1] == ref[1] and got[2] == ref[2]
 
 
+def test_select_ties_at_large_J_resolve_lexicographically(ampq):
+    """A case whose answer is known in closed form at a size no enumeration
+    reaches: 72 identical groups with columns (0, 0), (c, d), (c, d).  Every
+    choice of k groups in low precision gains the same, so the ordering rules
+    decide: smaller d cannot separate them either, and the lexicographically
+    smallest assignment puts column 1 (never its twin, column 2) in the LAST k
+    groups.  Dyadic values keep every sum exact."""
+    J, c, d = 72, 1.25, 0.5
+    c_tabs = [np.array([0.0, c, c])] * J
+    d_tabs = [np.array([0.0, d, d])] * J
+    for k in (0, 1, 7, 36, 71, 72):
+        p, ct, dt = ampq.select_tables(c_tabs, d_tabs, k * d + 0.25)
+        assert p.tolist() == [0] * (J - k) + [1] * k and ct == k * c and dt == k * d
+    # one group made slightly cheaper must be taken first; one made slightly more gainful too
+    d2 = [t.copy() for t in d_tabs]
+    d2[10] = np.array([0.0, d - 0.125, d])
+    p, ct, dt = ampq.select_tables(c_tabs, d2, 3 * d)
+    assert p.tolist() == [0] * 10 + [1] + [0] * (J - 13) + [1, 1] and dt == 3 * d - 0.125
+    c2 = [t.copy() for t in c_tabs]
+    c2[20] = np.array([0.0, c, c + 0.5])
+    p, ct, dt = ampq.select_tables(c2, d_tabs, 2 * d)
+    assert p.tolist() == [0] * 20 + [2] + [0] * (J - 22) + [1] and ct == 2 * c + 0.5
+
+
 def test_select_edge_cases(ampq):
     assert ampq.select_tables([[1.0]], [[2.0]], 1.0) is None
     p, c, d = ampq.select_tables([], [], 0.0)
