@@ -678,3 +678,87 @@ def test_shared_input_groups_score_in_one_read(ampq, orc, dtype, members):
     assert alone.get_pass_bytes()["score"] == 2 * members * xb + wb * (1 + R)
     shared.destroy()
     alone.destroy()
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_scores_with_every_option_mixed(ampq, orc, seed):
+    """Forty random scores per seed: 1-7 layers with random R, ragged sizes,
+    pointer offsets, inputs shared between layers, presets (zero included),
+    triangular operands, either scale mode, sharing on or off, any format list,
+    fp32 or bf16 -- every layer of every score against the oracle."""
+
+    class LT:
+        pass
+
+    tri = {T: torch.ones(T, T, dtype=torch.bool, device="cuda").triu(1) for T in (64, 128, 256)}
+    for it in range(40):
+        rng = np.random.default_rng(seed * 1000 + it)
+        gen = torch.Generator(device="cuda").manual_seed(seed * 1000 + it)
+        low = [[E4M3], [E5M2], [E4M3, E5M2], [E5M2, E4M3]][int(rng.integers(0, 4))]
+        dtype = torch.float32 if rng.random() < 0.4 else torch.bfloat16
+        pow2 = bool(rng.random() < 0.2)
+        ctx = _ctx(ampq, [0] + low)
+        if pow2:
+            ctx.set_scale_mode(ampq.SCALE_POW2)
+        if rng.random() < 0.2:
+            ctx.set_sharing(False)
+
+        def buf(n, std, off):
+            return torch.empty(n + 16, dtype=dtype, device="cuda").normal_(0, std, generator=gen)[off:off + n]
+
+        layers = []
+        for li in range(int(rng.integers(1, 8))):
+            R = int(rng.integers(1, 7))
+            nx = int(rng.choice([1, 7, 100, 4096, 8192, 32768, 50001, 65536, 150000, 300007]))
+            nw = int(rng.choice([0, 3, 1000, 32768, 70001, 131072]))
+            off = [int(o) for o in rng.choice([0, 0, 0, 1, 4, 8], 4)]
+            lt = LT()
+            lt.T = 0
+            shareable = [l for l in layers if not l.T]
+            if shareable and rng.random() < 0.45:    # reads the input of an earlier layer
+                src = shareable[int(rng.integers(0, len(shareable)))]
+                x, R = src.values[0], src.spec.R
+                nx = x.numel() // R
+            elif rng.random() < 0.2:                  # a stack of causal-softmax matrices
+                lt.T = int(rng.choice([64, 128, 256]))
+                H = int(rng.integers(1, 4))
+                nx = lt.T * lt.T * H
+                logits = torch.randn(R, H, lt.T, lt.T, generator=gen, device="cuda").masked_fill(tri[lt.T], float("-inf"))
+                x = torch.softmax(logits, -1).to(dtype).reshape(-1)
+            else:
+                x = buf(R * nx, 1.0, off[0])
+                if rng.random() < 0.3:
+                    x[int(rng.integers(0, x.numel()))] = float(rng.choice([100.0, -300.0, 1e-3]))
+            lt.spec = synth.LayerSpec("l%d" % li, synth.BGEMM if lt.T else synth.LINEAR, R, dtype,
+                                      synth.OperandSpec((R, nx), True), synth.OperandSpec((nw,), False))
+            lt.values = [x, buf(nw, 0.02, off[2])]
+            lt.grads = [buf(R * nx, 1e-3, off[1]).reshape(R, nx), buf(R * nw, 1e-3, off[3]).reshape(R, nw)]
+            lt.presets = [float(rng.choice([0.0, 0.5, 2.5, 1000.0])) if rng.random() < 0.2 else None,
+                          float(rng.choice([0.0, 0.01, 1.0])) if rng.random() < 0.15 else None]
+            layers.append(lt)
+        ids = []
+        for lt in layers:
+            lid = ctx.register_layer(lt.spec.kind, lt.spec.name, lt.spec.R)
+            code = ampq.torch_dtype_code(lt.values[1])
+            x, w = lt.values
+            ctx.bind_operand(lid, 0, code, x.data_ptr(), x.numel(), True, lt.grads[0].data_ptr(), x.numel() // lt.spec.R)
+            ctx.bind_operand(lid, 1, code, w.data_ptr(), w.numel(), False, lt.grads[1].data_ptr(), w.numel())
+            for k in range(2):
+                if lt.presets[k] is not None:
+                    ctx.set_amax(lid, k, lt.presets[k])
+            if lt.T:
+                ctx.set_causal(lid, 0, lt.T)
+            ids.append(lid)
+        ctx.score()
+        for lid, lt in zip(ids, layers):
+            ops = []
+            for k, op in enumerate((lt.spec.op0, lt.spec.op1)):
+                v, g = synth.to_numpy(lt.values[k]), synth.to_numpy(lt.grads[k])
+                a, sc, iv, seg = orc.score_operand(v.reshape(lt.spec.R, -1) if op.per_sample else v.reshape(-1),
+                                                   g.reshape(lt.spec.R, -1), lt.spec.R, op.per_sample, low,
+                                                   amax_preset=lt.presets[k], pow2=pow2)
+                ops.append(dict(amax=a, scale=sc, inv=iv, seg=seg))
+            ref = orc.layer_combine(ops[0]["seg"], ops[1]["seg"], [0] + low)
+            ref["ops"] = ops
+            compare_layer(ampq, ctx, lid, ref, 1 + len(low), "seed %d score %d layer %d" % (seed, it, lid))
+        ctx.destroy()
