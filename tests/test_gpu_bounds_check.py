@@ -1,8 +1,8 @@
 """The self-checking debug build (-DAMPQ_BOUNDS_CHECK): every scoring tile is
 checked against the extent of its tensor on the device and reported, not read,
 when it falls outside.  A mixed workload -- ragged and misaligned operands,
-shared weights with several sample groups, a triangular operand, streamed
-samples -- must pass the check and give, bit for bit, what the release build
+shared weights with several sample groups, inputs shared by several layers, a
+triangular operand, streamed samples -- must pass the check and give, bit for bit, what the release build
 gives.  Each build runs in a process of its own (AMPQ_LIBRARY picks it)."""
 import hashlib
 import os
@@ -29,6 +29,7 @@ def worker():
     ctx.set_formats([0, 1, 2])
     specs = synth.llama7b_block(16) + synth.attention_bgemm(8) + synth.toy_mlp(R=5, tokens=33, width=97, layers=2)
     lts = [synth.make_layer(s, "cuda", seed=21, layer=i) for i, s in enumerate(specs)]
+    synth.share_block_inputs(lts[:7])   # q, k, v and gate, up read one input each: scored as groups
     ids = []
     for lt in lts:
         lid = ctx.register_layer(lt.spec.kind, lt.spec.name, lt.spec.R)
