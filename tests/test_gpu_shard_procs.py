@@ -1,8 +1,11 @@
-"""Layer-sharded scoring by two processes that share the one GPU: each rank
-scores the layers `assign_layers` gives it with `ampq_score`, the ranks exchange
-the per-layer table over gloo (host tensors), and each runs the sub-graph sums
-and the selection.  Table and plan must equal those of a single process that
-scores everything, and the oracle's.  The two processes' kernels are independent
+"""Sharded scoring by two processes that share the one GPU, meeting over gloo
+(host tensors).  By layer: each rank scores the layers `assign_layers` gives it
+with `ampq_score`, the ranks exchange the per-layer table, and each runs the
+sub-graph sums and the selection.  By sample: each rank holds every layer but
+only its own calibration samples; the ranks exchange the per-tensor amax (MAX)
+between the amax pass and the scoring pass and merge their per-layer means
+afterwards.  Tables and plans must equal those of a single process that scores
+everything, and the oracle's.  The two processes' kernels are independent
 (nothing waits on the other process).  Run with -m gpu."""
 import json
 import os
@@ -79,6 +82,92 @@ def worker(rank, world, port, out):
         json.dump({"mine": mine, "table": table.tolist(), "res": res}, f)
 
 
+def _sample_specs():
+    from paper_2505_13060_b200 import synth
+
+    return synth.llama7b_block(32)[:4] + synth.toy_mlp(R=4, tokens=64, width=128, layers=2)
+
+
+def sample_worker(rank, world, port, out):
+    """Rank 0 holds sample 0, rank 1 samples 1..3 of every layer (R = 4)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_13060_b200 import binding, shard, synth
+
+    specs = _sample_specs()
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    r0, r1 = (0, 1) if rank == 0 else (1, 4)
+    ctx = binding.Context(0, torch.cuda.current_stream().cuda_stream)
+    ctx.set_formats([0, E4M3])
+    keep, ids = [], []
+    for i, sp in enumerate(specs):
+        lt = synth.make_layer(sp, "cuda", seed=17, layer=i)   # the same tensors on both ranks; each binds its samples
+        x, gx = lt.values[0][r0:r1].contiguous(), lt.grads[0][r0:r1].contiguous()
+        w, gw = lt.values[1], lt.grads[1][r0:r1].contiguous()
+        keep += [x, gx, w, gw]
+        lid = ctx.register_layer(sp.kind, sp.name, r1 - r0)
+        code = binding.torch_dtype_code(x)
+        ctx.bind_operand(lid, 0, code, x.data_ptr(), x.numel(), True, gx.data_ptr(), x.numel() // (r1 - r0))
+        ctx.bind_operand(lid, 1, code, w.data_ptr(), w.numel(), False, gw.data_ptr(), w.numel())
+        ids.append(lid)
+    ctx.measure_amax()
+    amax = shard.reduce_amax(np.stack([ctx.get_amax(i) for i in ids]))
+    for k, lid in enumerate(ids):
+        for op in range(2):
+            ctx.set_amax(lid, op, float(amax[k, op]))
+    ctx.score()
+    table = shard.merge_sample_rows(binding, ctx.get_layer_table(ids), r1 - r0)
+    ctx.destroy()
+    dist.barrier()
+    dist.destroy_process_group()
+    with open(os.path.join(out, "sample_rank%d.json" % rank), "w") as f:
+        json.dump({"amax": amax.tolist(), "table": table.tolist()}, f)
+
+
+def _spawn(tmp_path, mode):
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__), mode, str(r), "2", str(port), str(tmp_path)])
+             for r in range(2)]
+    for p in procs:
+        assert p.wait(timeout=600) == 0
+
+
+@pytest.mark.gpu
+def test_two_processes_score_their_samples_and_merge(tmp_path, ampq, orc):
+    import torch
+
+    from helpers import REL_TOL, compare_layer, oracle_layer
+    from paper_2505_13060_b200 import shard, synth
+
+    _spawn(tmp_path, "samples")
+    got = [json.load(open(tmp_path / ("sample_rank%d.json" % r))) for r in range(2)]
+    assert got[0] == got[1]   # both ranks end with the same amax and the same merged table, bit for bit
+    specs = _sample_specs()
+    one = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
+    one.set_formats([0, E4M3])
+    lts = [synth.make_layer(sp, "cuda", seed=17, layer=i) for i, sp in enumerate(specs)]
+    ids = []
+    for lt in lts:
+        lid = one.register_layer(lt.spec.kind, lt.spec.name, lt.spec.R)
+        ampq.bind_layer_tensors(one, lid, lt)
+        ids.append(lid)
+    one.score()
+    whole = one.get_layer_table(ids)
+    merged = np.array(got[0]["table"])
+    assert np.allclose(merged, whole, rtol=1e-12, atol=0)   # a mean of means against one mean: the order of additions
+    for k, (lid, lt) in enumerate(zip(ids, lts)):
+        ref = oracle_layer(orc, lt, [E4M3])
+        res = compare_layer(ampq, one, lid, ref, F, lt.spec.name)
+        assert res["amax"].tobytes() == np.array(got[0]["amax"][k], np.float32).tobytes()
+        want = shard.layer_row(ref, F)
+        assert np.all(np.abs(merged[k] - want) <= REL_TOL * np.abs(want))
+    one.destroy()
+
+
 @pytest.mark.gpu
 def test_two_processes_score_their_layers_and_meet_in_the_table(tmp_path, ampq, orc):
     import torch
@@ -86,14 +175,7 @@ def test_two_processes_score_their_layers_and_meet_in_the_table(tmp_path, ampq, 
     from helpers import REL_TOL, oracle_layer
     from paper_2505_13060_b200 import shard, synth
 
-    sock = socket.socket()
-    sock.bind(("127.0.0.1", 0))
-    port = sock.getsockname()[1]
-    sock.close()
-    procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__), str(r), "2", str(port), str(tmp_path)])
-             for r in range(2)]
-    for p in procs:
-        assert p.wait(timeout=600) == 0
+    _spawn(tmp_path, "layers")
     got = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in range(2)]
     specs = _specs()
     L = len(specs)
@@ -122,4 +204,5 @@ def test_two_processes_score_their_layers_and_meet_in_the_table(tmp_path, ampq, 
 if __name__ == "__main__":
     sys.path.insert(0, ROOT)
     sys.path.insert(0, os.path.join(ROOT, "tests"))
-    worker(int(sys.argv[1]), int(sys.argv[2]), int(sys.argv[3]), sys.argv[4])
+    fn = sample_worker if sys.argv[1] == "samples" else worker
+    fn(int(sys.argv[2]), int(sys.argv[3]), int(sys.argv[4]), sys.argv[5])
