@@ -221,6 +221,12 @@ int ampq_fake_quant(ampq_ctx *ctx, int dtype, int fmt, const void *values, long 
 /* Number of kernel launches issued by the last ampq_score (diagnostics). */
 int ampq_last_launch_count(const ampq_ctx *ctx);
 
+/* log2 of the scoring tile (elements) the last ampq_score used, 13..21: the
+ * largest that still gives every CTA of the persistent grid 16 tiles; 0 before
+ * a score (diagnostics: tests use it to check that they run the launch geometry
+ * they mean to). */
+int ampq_last_tile_shift(const ampq_ctx *ctx);
+
 /* Bytes of the bound tensors that the last ampq_score (or ampq_measure_amax)
  * reads (diagnostics; host pointer, bytes[2]): bytes[0] the amax pass -- every
  * operand without a preset once, an operand several layers share once;

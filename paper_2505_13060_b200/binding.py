@@ -38,7 +38,7 @@ EXPORTS = [
     "ampq_group_costs_table", "ampq_stream_begin", "ampq_stream_sample", "ampq_stream_end", "ampq_fake_quant",
     "ampq_partition", "ampq_gain_table", "ampq_select_in_order",
     "ampq_set_scale_mode", "ampq_measure_amax", "ampq_get_amax", "ampq_set_causal", "ampq_set_measured",
-    "ampq_set_sharing", "ampq_get_pass_bytes", "ampq_merge_sample_tables", "ampq_get_layer_table",
+    "ampq_set_sharing", "ampq_get_pass_bytes", "ampq_merge_sample_tables", "ampq_get_layer_table", "ampq_last_tile_shift",
 ]
 NOALLOC_MAX_NUMEL = 2147483648
 
@@ -75,6 +75,7 @@ def lib():
     L.ampq_set_amax.argtypes = [vp, i, i, C.c_float]
     L.ampq_score.argtypes = [vp]
     L.ampq_last_launch_count.argtypes = [vp]
+    L.ampq_last_tile_shift.argtypes = [vp]
     L.ampq_set_timing.argtypes = [vp, i]
     L.ampq_get_timing.argtypes = [vp, fp]
     L.ampq_get_layer.argtypes = [vp, i, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -323,6 +324,9 @@ class Context:
 
     def last_launch_count(self) -> int:
         return lib().ampq_last_launch_count(self._h)
+
+    def last_tile_shift(self) -> int:
+        return lib().ampq_last_tile_shift(self._h)
 
     def get_pass_bytes(self) -> dict:
         """Bytes of bound tensors the last pass reads: amax pass, scoring pass."""

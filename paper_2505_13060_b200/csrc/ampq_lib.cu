@@ -1104,6 +1104,8 @@ int ampq_fake_quant(ampq_ctx* ctx, int dtype, int fmt, const void* values, long 
 
 int ampq_last_launch_count(const ampq_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int ampq_last_tile_shift(const ampq_ctx* ctx) { return ctx && !ctx->dirty && !ctx->tens.empty() ? ctx->tile_shift : 0; }
+
 int ampq_get_pass_bytes(ampq_ctx* ctx, long long* bytes) {
     if (!ctx || !bytes) return AMPQ_ERR_INVALID;
     if (ctx->dirty || ctx->streaming || !(ctx->scored || ctx->amax_ready))

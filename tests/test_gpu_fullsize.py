@@ -36,18 +36,19 @@ def _same_as_block0(ctx, ids, per_block, blocks):
 def test_full_size_llama7b_block_whole(ampq, orc):
     """All 7 linear layers of one full-size Llama-7B-shaped block (R = 4 samples
     of 2048 tokens; 3.2 GB scored), every value against the oracle.  The block is
-    bound 16 times (as the benchmark binds resident slots, pointer sharing off)
-    so that the score uses the benchmark's 2^19-element tiles."""
+    bound 32 times (as the benchmark binds resident slots, pointer sharing off)
+    so that the score uses the tiles of the 32-block workload: 2^21 elements."""
     import bench
 
     _need(12)
     specs = bench.workload_specs("llama7b")
-    blocks = 16
+    blocks = 32
     ctx = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
     ctx.set_formats([0, E4M3, E5M2])
     slots, ids, scored = bench.bind_workload(ctx, specs, blocks, 1, torch.device("cuda", 0), seed=21)
     assert scored == blocks * sum(s.scored_bytes() for s in specs)
     ctx.score()
+    assert ctx.last_tile_shift() == 21
     for i, lt in enumerate(slots[0]):
         ref = oracle_layer(orc, lt, [E4M3, E5M2], threads=THREADS)
         compare_layer(ampq, ctx, ids[i], ref, 3, "7B block " + lt.spec.name)
@@ -59,8 +60,8 @@ def test_full_size_llama7b_block_whole(ampq, orc):
 @pytest.mark.parametrize("causal", [False, True])
 def test_full_size_attention_layer(ampq, orc, causal):
     """One full-size attention layer (Q,K and P,V with R = 4, 32 heads, T = 2048,
-    head size 128; P a causal softmax) bound 12 times so that the score takes the
-    largest tile: dense, and with the causal declaration (tiles of a matrix are
+    head size 128; P a causal softmax) bound 16 times so that the score takes the
+    largest tile (2^21 elements, as the 32-layer workload does): dense, and with the causal declaration (tiles of a matrix are
     then visited in rotated order and only the lower triangle is read).  Both
     against the oracle, which always scores the full operand; amax and scales bit
     for bit, FP8 codes of one (sample, head) slice of P bit for bit."""
@@ -68,11 +69,12 @@ def test_full_size_attention_layer(ampq, orc, causal):
 
     _need(10)
     specs = bench.workload_specs("attention")
-    blocks = 12
+    blocks = 16
     ctx = ampq.Context(0, torch.cuda.current_stream().cuda_stream)
     ctx.set_formats([0, E4M3])
     slots, ids, scored = bench.bind_workload(ctx, specs, blocks, 1, torch.device("cuda", 0), seed=22, causal=causal)
     ctx.score()
+    assert ctx.last_tile_shift() == 21   # a 2048 x 2048 matrix spans two tiles: the rotated visiting order is in play
     dense_bytes = blocks * sum(s.scored_bytes() for s in specs)
     assert scored < 0.6 * dense_bytes if causal else scored == dense_bytes
     pb = ctx.get_pass_bytes()

@@ -363,6 +363,7 @@ def test_full_size_llama70b_sampled_layers(ampq, orc):
     slots, ids, scored = bench.bind_workload(ctx, specs, blocks, nres, torch.device("cuda", 0), seed=7)
     assert len(ids) == 560 and scored == 614717194240
     ctx.score()
+    assert ctx.last_tile_shift() == 21
     names = [s.name for s in specs]
     for blk, name in ((0, "k"), (1, "o"), (1, "down")):
         i = names.index(name)
