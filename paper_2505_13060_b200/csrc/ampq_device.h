@@ -34,8 +34,8 @@ static_assert(kSubElems % (1 << kMinTileShift) == 0, "a flush block is a whole n
 static_assert(kAmaxTileElems >= (1 << 15), "an amax tile holds whole rows of the largest triangular matrix");
 constexpr int kMaxLow = 2;             // low-precision formats scored in one pass
 constexpr int kMaxAcc = 1 + kMaxLow;   // accumulators per segment: S, D_0, D_1
-constexpr int kMaxRB = 4;              // samples whose gradients share one read of shared values
-constexpr int kScoreClasses = 2 * kMaxRB + 2;  // scoring launches of one score: element type x samples per read,
+constexpr int kMaxRB = 4;              // gradient streams per read of the values: samples of a shared operand, or layers reading one input
+constexpr int kScoreClasses = 2 * kMaxRB + 2;  // scoring launches of one score: element type x streams per read,
                                                // plus one class per element type for causal (triangular) operands
 constexpr int kMinCausalShift = 6, kMaxCausalShift = 15;  // T between 64 and 32768
 

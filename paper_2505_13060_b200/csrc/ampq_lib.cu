@@ -126,7 +126,7 @@ struct ampq_ctx {
 
     // tables of the last score (host copies)
     std::vector<Tensor> tens;
-    // tile_begin[dtype * kMaxRB + rb - 1]: tiles of `dtype` operands scored with rb samples per read
+    // tile_begin[dtype * kMaxRB + rb - 1]: tiles of `dtype` operands scored with rb gradient streams per read
     std::vector<long long> tile_begin[kScoreClasses], amax_tile_begin;
     std::vector<Segment> segs;
     std::vector<Layer> lay;
