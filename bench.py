@@ -50,11 +50,10 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md (a 1.98 GB case;
 # traffic grows in proportion to the elements).  It holds only for the kernel
 # source it was taken on: `kernels_sha256` is the digest of ampq_kernels.cu +
-# ampq_device.h (at capture time, plus later edits to comments only), and the bench
-# reports traffic = null otherwise.
+# ampq_device.h at capture time, and the bench reports traffic = null otherwise.
 NCU_TRAFFIC = {
     "kernels_sha256": "504a1eb9e39bd496d4a1f1cbe80743bc420cea27dd48bcadf0ae52f374e98e0e",
-    "dram_bytes_per_scored_byte": {"e4m3": 1.0061},
+    "dram_bytes_per_scored_byte": {"e4m3": 1.0059},
     "source": "profiles/score_kernel_amax_kernel_llama70b_qkvo_ncu_full.md",
 }
 
